@@ -1,0 +1,370 @@
+#!/usr/bin/env python
+"""Benchmark of the Stochastic Attention hot path on B200.
+
+One step = one pass of the forward hot path over one batch of the Qwen3-8B-shaped
+workload (bf16, B=1, 32 query / 8 KV heads, d=128, n=32768, w=1024): a fresh permutation
+(sa_make_perm) followed by the gated SA+SWA forward (sa_swa_gated_forward), which runs the
+fused SA kernel, the plain SWA kernel and the gate.  `value` is tokens/s of that step.
+Beside it the JSON line reports the SA-only and SWA-only forward (tokens/s, TFLOP/s with
+4*B*Hq*n*w*d nominal flops, SA overhead over SWA), the permutation alone, the backward on
+the pre-training shape, a roofline entry for the SA forward kernel timed live with CUDA
+events inside the step, an end-to-end number with host buffers, and the float64 CPU oracle
+timed on a bounded sample.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload C3]
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "SA fwd tokens/s (step = fresh permutation + gated SA+SWA forward)"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        p["source"] = "measured"
+        return p
+    p = dict(FALLBACK_PEAKS)
+    p["source"] = "fallback"
+    return p
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, r[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def event_ms(fn, iters, warmup, torch):
+    """Mean milliseconds per call of fn, CUDA events on the current stream."""
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters
+
+
+def oracle_sample_rate(c, t, rows_count, seed=0):
+    """Times the float64 oracle (both branches + gate) on a random sample of query rows of
+    workload c; returns (tokens/s extrapolated to whole tokens, seconds, rows, threads)."""
+    import numpy as np
+
+    import oracle
+    from paper_2604_00754_b200.workloads import as_f64
+    q, k, v = as_f64(t["q"]), as_f64(t["k"]), as_f64(t["v"])
+    perm, inv = oracle.make_perm(c.seed, 0, c.B, c.n)
+    rng = np.random.default_rng(seed)
+    rows = np.sort(rng.choice(c.B * c.Hq * c.n, size=rows_count, replace=False)).astype(np.int64)
+    lg = t["gate_logits"].double().numpy()
+    t0 = time.perf_counter()
+    ysa, _ = oracle.forward_rows(0, q, k, v, perm, inv, c.w, c.flags, rows)
+    ysw, _ = oracle.forward_rows(1, q, k, v, None, None, c.w, c.flags, rows)
+    g = 1 / (1 + np.exp(-lg))
+    hq = (rows // c.n) % c.Hq
+    y = g[0, hq][:, None] * ysa + g[1, hq][:, None] * ysw
+    dt = time.perf_counter() - t0
+    assert np.isfinite(y).all()
+    tokens = rows_count / c.Hq          # a token is done when all its Hq rows are
+    return tokens / dt, dt, rows_count, oracle.n_threads()
+
+
+def run_reference(args, c):
+    """Reference arm: the CPU oracle as it stands, on host cores, bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2604_00754_b200 import workloads as wl
+    t = wl.draw(c)
+    rows = 32768
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample_rate(c, t, 1024)
+    rates, secs = [], []
+    for s in range(args.steps):
+        r, dt, _, threads = oracle_sample_rate(c, t, rows, seed=s)
+        rates.append(r)
+        secs.append(dt)
+    value = sum(rows / c.Hq for _ in rates) / sum(secs)
+    sample = "%d random query rows (of %d) per step, both branches + gate, extrapolated" % (
+        rows, c.B * c.Hq * c.n)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1e3 * sum(secs) / len(secs), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(c),
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": threads, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0,
+                "d2h_bytes_per_step": 0},
+    }))
+
+
+def workload_config(c):
+    return {"workload": c.name, "B": c.B, "Hq": c.Hq, "Hkv": c.Hkv, "n": c.n, "d": c.d, "w": c.w,
+            "flags": "causal(original order)+circular window; SWA branch one-sided",
+            "l2_policy": "inputs larger than L2 (Q+K+V+Y = %.0f MB per step)" % (
+                2 * (2 * c.B * c.Hq + 2 * c.B * c.Hkv) * c.n * c.d / 1e6)}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="C3")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the side measurements (SWA, backward, e2e, CPU oracle)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    from paper_2604_00754_b200 import workloads as wl
+    c = {k.split("_")[0]: v for k, v in wl.CONFIGS.items()}[args.workload]
+    if args.impl == "reference":
+        run_reference(args, c)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    from paper_2604_00754_b200 import binding as sa
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    sa.load_library()
+    pk = peaks()
+
+    # Each rank holds its own batch of independent sequences (the path shards over
+    # sequences and KV-head groups with no exchange step): weak scaling.
+    cr = c.scaled(seed=c.seed + rank)
+    host = wl.draw(cr, pin=True)
+    dev = {k: v.cuda(non_blocking=True) for k, v in host.items()}
+    q, k, v, lg = dev["q"], dev["k"], dev["v"], dev["gate_logits"]
+    perm = torch.empty(c.B, c.n, dtype=torch.int32, device="cuda")
+    inv = torch.empty_like(perm)
+    y = torch.empty_like(q)
+    prob = sa.SaProblem(B=c.B, n=c.n)
+    ws = torch.empty(sa.sa_workspace_bytes(prob, sa.OP_MAKE_PERM), dtype=torch.uint8, device="cuda")
+    out = {"y": y}
+    torch.cuda.synchronize()
+
+    layer = [0]
+
+    def step():
+        sa.sa_make_perm(cr.seed, layer[0], c.B, c.n, perm=perm, inv=inv, ws=ws)
+        sa.sa_swa_gated_forward(q, k, v, perm, inv, lg, c.w, c.flags, out=out)
+        layer[0] += 1
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    # timed region: K steps, the SA kernel of every step bracketed by its own event pair
+    pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+             for _ in range(args.steps)]
+    for a, b in pairs:
+        a.record(); b.record()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.25)
+    launches0 = sa.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for a, b in pairs:
+        sa.set_profile_events(a, b)
+        step()
+    e1.record()
+    barrier()
+    sa.set_profile_events(None, None)
+    launches = sa.launch_count() - launches0
+    clocks = sampler.stop()
+    total_ms = e0.elapsed_time(e1)
+    sa_kernel_ms = statistics.mean(a.elapsed_time(b) for a, b in pairs)
+    if world > 1:
+        tt = torch.tensor([total_ms], device="cuda")
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt.item())
+    assert sa.sa_read_status() == 0
+    ms_per_step = total_ms / args.steps
+    tokens_per_step = c.B * c.n * world
+    value = tokens_per_step / (ms_per_step * 1e-3)
+
+    flops_branch = 4.0 * c.B * c.Hq * c.n * c.w * c.d
+    achieved = flops_branch / (sa_kernel_ms * 1e-3) / 1e12
+    sustained = args.steps * ms_per_step > 1500.0
+    peak = pk["bf16_tflops_sustained"] if sustained else pk["bf16_tflops"]
+    line = {
+        "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic", "config": workload_config(c), "clocks": clocks,
+        "gpu_launches": int(launches),
+        "roofline": {"kernel": "fused SA forward (gather, QK^T, softmax, PV, scatter+gate)",
+                     "bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                     "frac": achieved / peak,
+                     "peak_kind": "%s bf16 %s" % (pk["source"], "sustained" if sustained else "burst"),
+                     "kernel_ms": sa_kernel_ms, "flops_per_launch": flops_branch,
+                     "traffic": None},
+    }
+
+    if rank == 0 and not args.no_extras:
+        line.update(extras(args, c, wl, sa, torch, dev, host, perm, inv, ws, y, pk))
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def extras(args, c, wl, sa, torch, dev, host, perm, inv, ws, y, pk):
+    """Side measurements on rank 0, outside the timed region of `value`."""
+    q, k, v, lg = dev["q"], dev["k"], dev["v"], dev["gate_logits"]
+    flops = 4.0 * c.B * c.Hq * c.n * c.w * c.d
+    it = max(5, args.steps // 2)
+    res = {}
+    sa_ms = event_ms(lambda: sa.sa_forward(q, k, v, perm, inv, c.w, c.flags, y=y), it, 3, torch)
+    swa_ms = event_ms(lambda: sa.sa_swa_forward(q, k, v, c.w, c.flags, y=y), it, 3, torch)
+    perm_ms = event_ms(lambda: sa.sa_make_perm(c.seed, 1, c.B, c.n, perm=perm, inv=inv, ws=ws),
+                       it, 3, torch)
+
+    def side(ms):
+        tf = flops / (ms * 1e-3) / 1e12
+        return {"ms": ms, "tokens_per_s": c.B * c.n / (ms * 1e-3), "tflops": tf,
+                "frac_of_burst": tf / pk["bf16_tflops"],
+                "frac_of_sustained": tf / pk["bf16_tflops_sustained"],
+                "frac_of_datasheet": tf / 2250.0}
+    res["sa_fwd"] = side(sa_ms)
+    res["swa_fwd"] = side(swa_ms)
+    res["sa_overhead_vs_swa"] = sa_ms / swa_ms - 1.0
+    res["make_perm_ms"] = perm_ms
+
+    # end to end: host (pinned) inputs -> device, the step, result back to the host
+    hy = torch.empty_like(host["q"]).pin_memory()
+    h2d = sum(host[n_].numel() * host[n_].element_size() for n_ in ("q", "k", "v", "gate_logits"))
+    d2h = hy.numel() * hy.element_size()
+    out = {"y": y}
+    layer = [1000]
+
+    def e2e_step():
+        for n_ in ("q", "k", "v", "gate_logits"):
+            dev[n_].copy_(host[n_], non_blocking=True)
+        sa.sa_make_perm(c.seed, layer[0], c.B, c.n, perm=perm, inv=inv, ws=ws)
+        sa.sa_swa_gated_forward(dev["q"], dev["k"], dev["v"], perm, inv, dev["gate_logits"], c.w,
+                                c.flags, out=out)
+        hy.copy_(y, non_blocking=True)
+        layer[0] += 1
+    e2e_ms = event_ms(e2e_step, it, 2, torch)
+    res["e2e"] = {"value": c.B * c.n / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms,
+                  "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+
+    # backward on the pre-training shape (fresh permutation, gated forward saving, backward)
+    c5 = wl.C5
+    t5 = {k_: v_.cuda() for k_, v_ in wl.draw(c5).items()}
+    p5, i5 = sa.sa_make_perm(c5.seed, 0, c5.B, c5.n)
+    saved = {}
+    bout = {}
+    bws = torch.empty(sa.sa_workspace_bytes(sa.make_problem(t5["q"], t5["k"], c5.w, c5.flags),
+                                            sa.OP_BACKWARD), dtype=torch.uint8, device="cuda")
+
+    def fwd5():
+        r = sa.sa_swa_gated_forward(t5["q"], t5["k"], t5["v"], p5, i5, t5["gate_logits"], c5.w,
+                                    c5.flags, save_for_bwd=True, out=saved)
+        saved.update(zip(("y", "y_sa", "y_swa", "lse_sa", "lse_swa"), r))
+
+    def bwd5():
+        r = sa.sa_backward(t5["q"], t5["k"], t5["v"], p5, i5, t5["gate_logits"], saved["y_sa"],
+                           saved["y_swa"], saved["lse_sa"], saved["lse_swa"], t5["dy"], c5.w,
+                           c5.flags, ws=bws, out=bout)
+        bout.update(zip(("dq", "dk", "dv", "dgate"), r))
+    f5 = event_ms(fwd5, it, 2, torch)
+    b5 = event_ms(bwd5, it, 2, torch)
+    fl5 = 2 * 4.0 * c5.B * c5.Hq * c5.n * c5.w * c5.d
+    res["pretrain_layer_C5"] = {
+        "gated_fwd_ms": f5, "bwd_ms": b5, "tokens_per_s_fwd_bwd": c5.B * c5.n / ((f5 + b5) * 1e-3),
+        "tflops_fwd_bwd": 3.5 * fl5 / ((f5 + b5) * 1e-3) / 1e12}
+    del t5, saved, bout, bws
+    torch.cuda.empty_cache()
+
+    rate, dt, rows, threads = oracle_sample_rate(c, host, 196608)
+    res["cpu_baseline"] = {
+        "value": rate, "unit": "tokens/s", "cores": threads, "kind": "oracle",
+        "sample": "%d random query rows of %d (both branches + gate), %.1f s, extrapolated to "
+                  "whole tokens" % (rows, c.B * c.Hq * c.n, dt)}
+    return res
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,172 @@
+/*
+ * sa.h -- C ABI of the Stochastic Attention (SA) hot path for NVIDIA B200 (sm_100a).
+ *
+ * The operation (paper Sec. 3.3, Alg. 1, Eq. 3/4; App. B "Stochastic attention mask"):
+ * draw a uniform random permutation sigma of the n tokens of a sequence, run softmax
+ * sliding-window attention of width w in the permuted order, and put the result back
+ * in the original order.  In the original order, query token i sees key token j iff
+ *
+ *     2 * dist(inv[i], inv[j]) < w        (window in shuffled space, Eq. 3)
+ *     and, with SA_CAUSAL,  j <= i        (causality in ORIGINAL space, App. B)
+ *
+ * where inv[i] is the slot of token i (the paper's sigma(i)), perm[p] the token in
+ * slot p, and dist is the circular distance |a-b|_n = min(|a-b|, n-|a-b|) of Sec. 3.1
+ * (plain |a-b| with SA_LINEAR_WINDOW).  The gated form (Sec. 3.4, Eq. 5, Alg. 2) adds
+ * an ordinary sliding-window branch: y = sig(l_sa) y_sa + sig(l_swa) y_swa, with two
+ * independent sigmoids and, in this library, one scalar logit per head and branch.
+ *
+ * General conventions
+ *   - Every pointer is a DEVICE pointer unless a comment says "host".  The caller owns
+ *     every buffer, workspace included; the library allocates nothing and frees nothing.
+ *   - Work is only enqueued on the caller's stream; no call synchronises except
+ *     sa_read_status.  Inputs are never written.
+ *   - Tensors: q, y, dq, dy, y_sa, y_swa are [B,Hq,n,d]; k, v, dk, dv are [B,Hkv,n,d];
+ *     addressed through the element strides in sa_problem (d is contiguous).  perm and
+ *     inv are contiguous int32 [B,n]; lse_* contiguous fp32 [B,Hq,n]; gate logits
+ *     contiguous fp32 [2,Hq] (row 0 = SA branch, row 1 = SWA branch).
+ *   - Everything the caller sees is in ORIGINAL token order.
+ *   - Query head hq reads KV head hq / (Hq/Hkv) (contiguous GQA groups).
+ *   - Data pointers must be 16-byte aligned and all strides multiples of 8 elements.
+ *   - Errors the host can see (bad shapes, null or misaligned pointers, short
+ *     workspace) return a code before anything is launched.  Errors only the device can
+ *     see (SA_VALIDATE_PERM found a non-bijection, a bounded wait ran out) are recorded
+ *     in a device status word that sa_read_status returns; the kernel then returns
+ *     normally and its outputs are unspecified.  Nothing traps.
+ */
+#ifndef SA_B200_SA_H_
+#define SA_B200_SA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct CUstream_st* sa_stream_t; /* a cudaStream_t; NULL = the legacy default stream */
+
+typedef enum {
+  SA_OK = 0,
+  SA_ERR_INVALID_ARG = 1, /* null/misaligned pointer, bad shape or stride               */
+  SA_ERR_UNSUPPORTED = 2, /* valid request this build has no kernel for                 */
+  SA_ERR_WORKSPACE = 3,   /* ws_bytes smaller than sa_workspace_bytes()                  */
+  SA_ERR_CUDA = 4,        /* a CUDA runtime call failed (launch error, no device)       */
+  SA_ERR_BAD_PERM = 5,    /* device: perm/inv are not mutually inverse bijections       */
+  SA_ERR_TIMEOUT = 6      /* device: a bounded wait inside a kernel ran out             */
+} sa_status;
+
+typedef enum { SA_F32 = 0, SA_BF16 = 1 } sa_dtype;
+
+enum {
+  SA_CAUSAL = 1,        /* j <= i in the original order (Sec. 3.3 causal paragraph; App. B)   */
+  SA_LINEAR_WINDOW = 2, /* plain |a-b| between slots; default is circular |a-b|_n (Sec. 3.1) */
+  SA_SWA_ONE_SIDED = 4, /* the SWA branch uses {j : 0 <= i-j <= w-1} (Sec. 3.1 footnote);    */
+                        /* without it the SWA branch is the SA rule under the identity       */
+  SA_SAVE_FOR_BWD = 8,  /* gated forward: y_sa, y_swa, lse_sa, lse_swa must all be given     */
+  SA_VALIDATE_PERM = 16 /* check on the device that inv[perm[p]] == p, 0 <= perm[p] < n      */
+};
+
+typedef enum {
+  SA_OP_MAKE_PERM = 0,
+  SA_OP_FORWARD = 1,
+  SA_OP_SWA_FORWARD = 2,
+  SA_OP_GATED_FORWARD = 3,
+  SA_OP_BACKWARD = 4,
+  SA_OP_COVERAGE = 5
+} sa_op;
+
+typedef struct {
+  int32_t B, Hq, Hkv;  /* batch, query heads, KV heads; Hq % Hkv == 0                     */
+  int32_t n, d, w;     /* tokens, head dim (multiple of 8, <= 256), window width (>= 1)   */
+  int32_t dtype;       /* sa_dtype of q/k/v/y/dy/dq/dk/dv                                 */
+  uint32_t flags;      /* SA_* bits                                                       */
+  float softmax_scale; /* multiplies q.k (Eq. 1); 0 selects 1/sqrt(d)                     */
+  int32_t L;           /* layers, used by SA_OP_COVERAGE sizing only; else ignored        */
+  int64_t q_stride[3];  /* element strides of q, y, dq, dy, y_sa, y_swa: batch, head, token */
+  int64_t kv_stride[3]; /* element strides of k, v, dk, dv: batch, head, token            */
+} sa_problem;
+
+/* Fills the two stride triples for contiguous [B,H,n,d] tensors.  Host-only helper. */
+void sa_problem_set_contiguous(sa_problem* p);
+
+/* Bytes of workspace the given operation needs for this problem (0 is possible; then
+ * ws may be NULL).  Only B, n matter for SA_OP_MAKE_PERM; L, n for SA_OP_COVERAGE.
+ * Returns (size_t)-1 for an invalid problem. */
+size_t sa_workspace_bytes(const sa_problem* p, int op);
+
+/* Alg. 1 line 1: one uniform random permutation per sequence and its inverse.
+ * Sequence b, token i gets the 64-bit key formed by the first two output words of
+ * Philox4x32-10 with counter (i, b, layer, 0) and key (seed low word, seed high word);
+ * perm[b,:] lists the tokens in increasing (key, token) order; inv[b, perm[b,p]] = p.
+ * A pure function of (seed, layer, b, n): any process regenerates the same sigma.
+ * perm, inv: out, int32 [B,n].  ws: scratch of sa_workspace_bytes(.., SA_OP_MAKE_PERM). */
+sa_status sa_make_perm(uint64_t seed, uint32_t layer, int32_t B, int32_t n, int32_t* perm,
+                       int32_t* inv, void* ws, size_t ws_bytes, sa_stream_t stream);
+
+/* SA forward (Alg. 1; Eq. 1 on the neighbourhood of Eq. 3; mask of App. B).
+ * Rows of q/k/v are gathered through perm inside the kernel and rows of y are scattered
+ * back; no permuted copy of any tensor is made.  y: out.  lse: out, nullable, the
+ * log-sum-exp of each query's visible scaled scores (needed by sa_backward). */
+sa_status sa_forward(const sa_problem* p, const void* q, const void* k, const void* v,
+                     const int32_t* perm, const int32_t* inv, void* y, float* lse, void* ws,
+                     size_t ws_bytes, sa_stream_t stream);
+
+/* Plain sliding-window attention in the original order (Eq. 1): the local branch of the
+ * gated form and the baseline the permutation overhead is measured against. */
+sa_status sa_swa_forward(const sa_problem* p, const void* q, const void* k, const void* v,
+                         void* y, float* lse, void* ws, size_t ws_bytes, sa_stream_t stream);
+
+/* Gated SA + SWA forward (Alg. 2, Eq. 5) with per-head scalar gates:
+ * y = sigmoid(gate_logits[0,hq]) * y_sa + sigmoid(gate_logits[1,hq]) * y_swa.
+ * y: out.  y_sa, y_swa, lse_sa, lse_swa: out, nullable unless SA_SAVE_FOR_BWD; the
+ * branch outputs are stored in the run dtype before they are combined. */
+sa_status sa_swa_gated_forward(const sa_problem* p, const void* q, const void* k,
+                               const void* v, const int32_t* perm, const int32_t* inv,
+                               const float* gate_logits, void* y, void* y_sa, void* y_swa,
+                               float* lse_sa, float* lse_swa, void* ws, size_t ws_bytes,
+                               sa_stream_t stream);
+
+/* Backward of sa_forward (gate_logits == NULL: y_swa, lse_swa, dgate_logits ignored, y_sa
+ * is the forward's y) or of sa_swa_gated_forward.  The paper only times this pass
+ * (Sec. 4.3); the formulas are the derivative of Eq. 1 / Eq. 5 with sigma constant:
+ *   P_ij = exp(scale q_i.k_j - lse_i), D_i = dY_x[i].Y_x[i], dV_j += P_ij dY_x[i],
+ *   dS_ij = P_ij (dY_x[i].V_j - D_i), dQ_i += scale dS_ij K_j, dK_j += scale dS_ij Q_i,
+ * per branch x with dY_x = g_x dY; dk, dv are summed over the query heads of a group;
+ * dgate_logits[x,hq] = g_x (1 - g_x) sum_{b,i,c} dY Y_x.   dq, dk, dv, dgate_logits: out. */
+sa_status sa_backward(const sa_problem* p, const void* q, const void* k, const void* v,
+                      const int32_t* perm, const int32_t* inv, const float* gate_logits,
+                      const void* y_sa, const void* y_swa, const float* lse_sa,
+                      const float* lse_swa, const void* dy, void* dq, void* dk, void* dv,
+                      float* dgate_logits, void* ws, size_t ws_bytes, sa_stream_t stream);
+
+/* Mask statistics over L layers, each with its own permutation (perm, inv int32 [L,n]):
+ * row_count[l,i] = number of keys query i sees at layer l (nullable), nnz[l] = their sum
+ * (int64 [L]); reach[l] = |R_{l+1}(src)|, the set reachable from token src through layers
+ * 0..l (Prop. 2: R_0 = {src}, R_{l+1} = union of the visible sets of R_l's members).
+ * Only n, w and the mask bits of flags are used. */
+sa_status sa_coverage(int32_t L, int32_t n, int32_t w, uint32_t flags, const int32_t* perm,
+                      const int32_t* inv, int32_t src, int64_t* nnz, int32_t* row_count,
+                      int32_t* reach, void* ws, size_t ws_bytes, sa_stream_t stream);
+
+/* Synchronises the stream, returns the device status word (SA_OK, SA_ERR_BAD_PERM or
+ * SA_ERR_TIMEOUT) of the current device and clears it. */
+sa_status sa_read_status(sa_stream_t stream);
+
+/* Static, human-readable name of a status code.  Host pointer. */
+const char* sa_status_string(sa_status s);
+
+/* Profiling hook.  start/stop are cudaEvent_t handles (host values) or both NULL.  While set,
+ * every SA-branch attention kernel launched by sa_forward / sa_swa_gated_forward is bracketed
+ * by cudaEventRecord(start) and cudaEventRecord(stop) on the call's stream, so a caller can
+ * time that one kernel inside a longer step.  Process-wide; not thread-safe.  The paper has
+ * no counterpart: this exists for the roofline measurement only. */
+void sa_set_profile_events(void* start, void* stop);
+
+/* Number of kernel launches this process has enqueued through the library so far
+ * (all entry points together); used by the benchmark's launch count. */
+uint64_t sa_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SA_B200_SA_H_ */

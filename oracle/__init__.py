@@ -225,3 +225,24 @@ def coverage(perm, inv, w, flags, src):
                             row_count.ctypes.data_as(ctypes.c_void_p),
                             reach.ctypes.data_as(ctypes.c_void_p))
     return nnz, row_count, reach
+
+
+def forward_rows(swa, q, k, v, perm, inv, w, flags, rows, scale=0.0):
+    """Eq. 1 for selected rows only; rows = flat (b*Hq+hq)*n+i indices.  Returns (y_rows, lse_rows)."""
+    q, qp = _f64(q)
+    k, kp = _f64(k)
+    v, vp = _f64(v)
+    B, Hq, n, d = q.shape
+    Hkv = k.shape[1]
+    perm, pp = _i32(None if swa else perm)
+    inv, ip = _i32(None if swa else inv)
+    rows = np.ascontiguousarray(rows, dtype=np.int64)
+    y = np.empty((rows.size, d), np.float64)
+    lse = np.empty(rows.size, np.float64)
+    _load().oracle_forward_rows(
+        ctypes.c_int32(int(swa)), ctypes.c_int32(B), ctypes.c_int32(Hq), ctypes.c_int32(Hkv),
+        ctypes.c_int32(n), ctypes.c_int32(d), ctypes.c_int32(w), ctypes.c_uint32(flags),
+        ctypes.c_double(_scale(d, scale)), qp, kp, vp, pp, ip, ctypes.c_int64(rows.size),
+        rows.ctypes.data_as(ctypes.c_void_p), y.ctypes.data_as(ctypes.c_void_p),
+        lse.ctypes.data_as(ctypes.c_void_p))
+    return y, lse

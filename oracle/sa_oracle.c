@@ -382,3 +382,37 @@ void oracle_coverage(int32_t L, int32_t n, int32_t w, uint32_t flags, const int3
   }
   free(cur); free(nxt);
 }
+
+/* Selected rows only: rows[t] is a flat (b*Hq + hq)*n + i index; y_rows [n_rows,d],
+ * lse_rows [n_rows].  Same arithmetic as oracle_forward, for spot checks at sizes where
+ * the whole tensor would take hours.                                             */
+void oracle_forward_rows(int32_t swa, int32_t B, int32_t Hq, int32_t Hkv, int32_t n, int32_t d,
+                         int32_t w, uint32_t flags, double scale, const double* q,
+                         const double* k, const double* v, const int32_t* perm,
+                         const int32_t* inv, int64_t n_rows, const int64_t* rows,
+                         double* y_rows, double* lse_rows) {
+  const int32_t G = Hq / Hkv;
+  (void)B;
+#pragma omp parallel
+  {
+    int32_t* cand = (int32_t*)malloc(sizeof(int32_t) * (size_t)n);
+    double* s_buf = (double*)malloc(sizeof(double) * (size_t)n);
+#pragma omp for schedule(dynamic, 16)
+    for (int64_t t = 0; t < n_rows; ++t) {
+      const int64_t r = rows[t];
+      const int32_t i = (int32_t)(r % n);
+      const int32_t hq = (int32_t)((r / n) % Hq);
+      const int32_t b = (int32_t)(r / ((int64_t)n * Hq));
+      const int32_t hk = hq / G;
+      const int32_t* pb = perm ? perm + (size_t)b * n : NULL;
+      const int32_t* ib = inv ? inv + (size_t)b * n : NULL;
+      const int32_t nc = collect_visible(swa, 0, n, w, flags, pb, ib, i, cand);
+      const double* kh = k + ((size_t)b * Hkv + hk) * n * d;
+      const double* vh = v + ((size_t)b * Hkv + hk) * n * d;
+      const double l = attend_row(d, scale, q + (size_t)r * d, kh, vh, cand, nc, s_buf,
+                                  y_rows + (size_t)t * d);
+      if (lse_rows) lse_rows[t] = l;
+    }
+    free(cand); free(s_buf);
+  }
+}

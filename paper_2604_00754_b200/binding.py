@@ -1,0 +1,282 @@
+"""Python binding of the C ABI declared in ``include/sa.h``: argument marshalling only.
+
+Every step of the path runs in the CUDA library; torch is used here for device memory
+and the current stream.  There is no fallback of any kind: if the shared library is
+missing and cannot be built, or a call returns an error status, an exception is raised.
+
+The functions carry the C names (``sa_make_perm``, ``sa_forward``, ``sa_swa_forward``,
+``sa_swa_gated_forward``, ``sa_backward``, ``sa_coverage``) and take torch CUDA tensors
+where the C functions take device pointers.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+from . import build as _build
+
+SA_OK = 0
+CAUSAL, LINEAR_WINDOW, SWA_ONE_SIDED, SAVE_FOR_BWD, VALIDATE_PERM = 1, 2, 4, 8, 16
+OP_MAKE_PERM, OP_FORWARD, OP_SWA_FORWARD, OP_GATED_FORWARD, OP_BACKWARD, OP_COVERAGE = range(6)
+F32, BF16 = 0, 1
+
+EXPORTS = [
+    "sa_problem_set_contiguous", "sa_workspace_bytes", "sa_make_perm", "sa_forward",
+    "sa_swa_forward", "sa_swa_gated_forward", "sa_backward", "sa_coverage", "sa_read_status",
+    "sa_status_string", "sa_launch_count", "sa_set_profile_events",
+]
+
+
+class SaProblem(ctypes.Structure):
+    _fields_ = [
+        ("B", ctypes.c_int32), ("Hq", ctypes.c_int32), ("Hkv", ctypes.c_int32),
+        ("n", ctypes.c_int32), ("d", ctypes.c_int32), ("w", ctypes.c_int32),
+        ("dtype", ctypes.c_int32), ("flags", ctypes.c_uint32),
+        ("softmax_scale", ctypes.c_float), ("L", ctypes.c_int32),
+        ("q_stride", ctypes.c_int64 * 3), ("kv_stride", ctypes.c_int64 * 3),
+    ]
+
+
+class SaError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s failed: %s (status %d)" % (where, status_string(status), status))
+
+
+_lib = None
+
+
+def load_library(path: Optional[str] = None) -> ctypes.CDLL:
+    """Loads (building first if the sources are newer) the CUDA library; raises if it cannot."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    if path is None:
+        path = _build.LIB
+        if _build.stale():
+            try:
+                _build.build_library()
+            except Exception as e:  # no nvcc, compile error
+                if not os.path.exists(path):
+                    raise RuntimeError("CUDA library %s is missing and could not be built: %s"
+                                       % (path, e)) from e
+    lib = ctypes.CDLL(path)
+    vp, i32, u32, u64, sz = (ctypes.c_void_p, ctypes.c_int32, ctypes.c_uint32, ctypes.c_uint64,
+                             ctypes.c_size_t)
+    pp = ctypes.POINTER(SaProblem)
+    lib.sa_problem_set_contiguous.argtypes = [pp]
+    lib.sa_problem_set_contiguous.restype = None
+    lib.sa_workspace_bytes.argtypes = [pp, ctypes.c_int]
+    lib.sa_workspace_bytes.restype = sz
+    lib.sa_make_perm.argtypes = [u64, u32, i32, i32, vp, vp, vp, sz, vp]
+    lib.sa_forward.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.sa_swa_forward.argtypes = [pp, vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.sa_swa_gated_forward.argtypes = [pp] + [vp] * 12 + [sz, vp]
+    lib.sa_backward.argtypes = [pp] + [vp] * 16 + [sz, vp]
+    lib.sa_coverage.argtypes = [i32, i32, i32, u32, vp, vp, i32, vp, vp, vp, vp, sz, vp]
+    lib.sa_read_status.argtypes = [vp]
+    for f in ("sa_make_perm", "sa_forward", "sa_swa_forward", "sa_swa_gated_forward",
+              "sa_backward", "sa_coverage", "sa_read_status"):
+        getattr(lib, f).restype = ctypes.c_int
+    lib.sa_status_string.argtypes = [ctypes.c_int]
+    lib.sa_status_string.restype = ctypes.c_char_p
+    lib.sa_set_profile_events.argtypes = [vp, vp]
+    lib.sa_set_profile_events.restype = None
+    lib.sa_launch_count.argtypes = []
+    lib.sa_launch_count.restype = u64
+    if path == _build.LIB:
+        _lib = lib
+    return lib
+
+
+def status_string(status: int) -> str:
+    return load_library().sa_status_string(int(status)).decode()
+
+
+def launch_count() -> int:
+    return int(load_library().sa_launch_count())
+
+
+def set_profile_events(start: Optional[torch.cuda.Event], stop: Optional[torch.cuda.Event]):
+    """Brackets the SA-branch attention kernel of later forward calls with these events."""
+    lib = load_library()
+    if start is None or stop is None:
+        lib.sa_set_profile_events(None, None)
+        return
+    # torch creates the underlying cudaEvent lazily, at the first record
+    if not start.cuda_event:
+        start.record()
+    if not stop.cuda_event:
+        stop.record()
+    lib.sa_set_profile_events(ctypes.c_void_p(start.cuda_event), ctypes.c_void_p(stop.cuda_event))
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(status: int, where: str):
+    if status != SA_OK:
+        raise SaError(status, where)
+
+
+def make_problem(q: torch.Tensor, k: torch.Tensor, w: int, flags: int, scale: float = 0.0,
+                 L: int = 0) -> SaProblem:
+    """Describes [B,H,n,d] tensors (any strides with d contiguous) to the library."""
+    if q.dtype == torch.float32:
+        dt = F32
+    elif q.dtype == torch.bfloat16:
+        dt = BF16
+    else:
+        raise TypeError("q/k/v must be float32 or bfloat16")
+    B, Hq, n, d = q.shape
+    p = SaProblem(B=B, Hq=Hq, Hkv=k.shape[1], n=n, d=d, w=int(w), dtype=dt, flags=int(flags),
+                  softmax_scale=float(scale), L=int(L))
+    if q.stride(3) != 1 or k.stride(3) != 1:
+        raise ValueError("the head dimension must be contiguous")
+    p.q_stride[:] = [q.stride(0), q.stride(1), q.stride(2)]
+    p.kv_stride[:] = [k.stride(0), k.stride(1), k.stride(2)]
+    return p
+
+
+def sa_workspace_bytes(p: SaProblem, op: int) -> int:
+    r = int(load_library().sa_workspace_bytes(ctypes.byref(p), int(op)))
+    if r == ctypes.c_size_t(-1).value:
+        raise SaError(1, "sa_workspace_bytes")
+    return r
+
+
+def _workspace(nbytes: int, device, ws: Optional[torch.Tensor]):
+    if ws is not None:
+        return ws
+    return torch.empty(max(nbytes, 16), dtype=torch.uint8, device=device)
+
+
+def _same_layout(ref: torch.Tensor, *others):
+    for t in others:
+        if t is not None and (t.shape != ref.shape or t.stride() != ref.stride()
+                              or t.dtype != ref.dtype):
+            raise ValueError("tensor does not share the layout of its reference tensor")
+
+
+def sa_make_perm(seed: int, layer: int, B: int, n: int, device="cuda", perm=None, inv=None,
+                 ws=None):
+    """One uniform permutation per sequence and its inverse (int32 [B,n] each)."""
+    lib = load_library()
+    perm = torch.empty(B, n, dtype=torch.int32, device=device) if perm is None else perm
+    inv = torch.empty(B, n, dtype=torch.int32, device=device) if inv is None else inv
+    p = SaProblem(B=B, n=n)
+    nbytes = sa_workspace_bytes(p, OP_MAKE_PERM)
+    ws = _workspace(nbytes, perm.device, ws)
+    _check(lib.sa_make_perm(int(seed) & (2 ** 64 - 1), int(layer), B, n, _ptr(perm), _ptr(inv),
+                            _ptr(ws), ws.numel(), _stream()), "sa_make_perm")
+    return perm, inv
+
+
+def sa_forward(q, k, v, perm, inv, w, flags=CAUSAL, scale=0.0, y=None, want_lse=False,
+               lse=None):
+    """SA forward; returns y (and lse when asked)."""
+    lib = load_library()
+    _same_layout(k, v)
+    p = make_problem(q, k, w, flags, scale)
+    y = torch.empty_like(q) if y is None else y
+    _same_layout(q, y)
+    if want_lse and lse is None:
+        lse = torch.empty(q.shape[:3], dtype=torch.float32, device=q.device)
+    _check(lib.sa_forward(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(perm), _ptr(inv),
+                          _ptr(y), _ptr(lse), None, 0, _stream()), "sa_forward")
+    return (y, lse) if (want_lse or lse is not None) else y
+
+
+def sa_swa_forward(q, k, v, w, flags=CAUSAL | SWA_ONE_SIDED, scale=0.0, y=None, want_lse=False,
+                   lse=None):
+    """Plain sliding-window attention forward in the original order."""
+    lib = load_library()
+    _same_layout(k, v)
+    p = make_problem(q, k, w, flags, scale)
+    y = torch.empty_like(q) if y is None else y
+    _same_layout(q, y)
+    if want_lse and lse is None:
+        lse = torch.empty(q.shape[:3], dtype=torch.float32, device=q.device)
+    _check(lib.sa_swa_forward(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(y), _ptr(lse),
+                              None, 0, _stream()), "sa_swa_forward")
+    return (y, lse) if (want_lse or lse is not None) else y
+
+
+def sa_swa_gated_forward(q, k, v, perm, inv, gate_logits, w, flags=CAUSAL | SWA_ONE_SIDED,
+                         scale=0.0, save_for_bwd=False, out=None):
+    """Gated SA + SWA forward.  Returns y, or (y, y_sa, y_swa, lse_sa, lse_swa) when saving.
+
+    ``out`` may hold preallocated tensors under the keys y, y_sa, y_swa, lse_sa, lse_swa."""
+    lib = load_library()
+    _same_layout(k, v)
+    out = dict(out or {})
+    if save_for_bwd:
+        flags |= SAVE_FOR_BWD
+        for name in ("y_sa", "y_swa"):
+            out.setdefault(name, torch.empty_like(q))
+        for name in ("lse_sa", "lse_swa"):
+            out.setdefault(name, torch.empty(q.shape[:3], dtype=torch.float32, device=q.device))
+    y = out.setdefault("y", torch.empty_like(q))
+    _same_layout(q, y, out.get("y_sa"), out.get("y_swa"))
+    p = make_problem(q, k, w, flags, scale)
+    _check(lib.sa_swa_gated_forward(
+        ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(perm), _ptr(inv), _ptr(gate_logits),
+        _ptr(y), _ptr(out.get("y_sa")), _ptr(out.get("y_swa")), _ptr(out.get("lse_sa")),
+        _ptr(out.get("lse_swa")), None, 0, _stream()), "sa_swa_gated_forward")
+    if save_for_bwd:
+        return y, out["y_sa"], out["y_swa"], out["lse_sa"], out["lse_swa"]
+    return y
+
+
+def sa_backward(q, k, v, perm, inv, gate_logits, y_sa, y_swa, lse_sa, lse_swa, dy, w,
+                flags=CAUSAL | SWA_ONE_SIDED, scale=0.0, ws=None, out=None):
+    """Backward of the (gated) forward.  Returns (dq, dk, dv, dgate_logits or None)."""
+    lib = load_library()
+    _same_layout(k, v)
+    _same_layout(q, dy, y_sa, y_swa)
+    out = dict(out or {})
+    dq = out.setdefault("dq", torch.empty_like(q))
+    dk = out.setdefault("dk", torch.empty_like(k))
+    dv = out.setdefault("dv", torch.empty_like(v))
+    _same_layout(q, dq)
+    _same_layout(k, dk, dv)
+    dgate = None
+    if gate_logits is not None:
+        dgate = out.setdefault("dgate", torch.empty(2, q.shape[1], dtype=torch.float32,
+                                                    device=q.device))
+    p = make_problem(q, k, w, flags, scale)
+    ws = _workspace(sa_workspace_bytes(p, OP_BACKWARD), q.device, ws)
+    _check(lib.sa_backward(
+        ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(perm), _ptr(inv), _ptr(gate_logits),
+        _ptr(y_sa), _ptr(y_swa), _ptr(lse_sa), _ptr(lse_swa), _ptr(dy), _ptr(dq), _ptr(dk),
+        _ptr(dv), _ptr(dgate), _ptr(ws), ws.numel(), _stream()), "sa_backward")
+    return dq, dk, dv, dgate
+
+
+def sa_coverage(perm, inv, w, flags, src, want_row_count=True, ws=None):
+    """Mask row counts, their totals, and reachable-set sizes over the L layers of perm [L,n]."""
+    lib = load_library()
+    L, n = perm.shape
+    dev = perm.device
+    nnz = torch.empty(L, dtype=torch.int64, device=dev)
+    reach = torch.empty(L, dtype=torch.int32, device=dev)
+    rc = torch.empty(L, n, dtype=torch.int32, device=dev) if want_row_count else None
+    p = SaProblem(n=n, L=L)
+    ws = _workspace(sa_workspace_bytes(p, OP_COVERAGE), dev, ws)
+    _check(lib.sa_coverage(L, n, int(w), int(flags), _ptr(perm), _ptr(inv), int(src), _ptr(nnz),
+                           _ptr(rc), _ptr(reach), _ptr(ws), ws.numel(), _stream()),
+           "sa_coverage")
+    return nnz, rc, reach
+
+
+def sa_read_status() -> int:
+    """Synchronises the current stream and returns (and clears) the device status word."""
+    return int(load_library().sa_read_status(_stream()))

@@ -1,0 +1,357 @@
+"""GPU parity: every entry point of the C ABI against the float64 CPU oracle on the
+same seeded inputs.  Integers bit-exact; fp32 outputs within 1e-4 max-abs; bf16 outputs
+within 2e-2 of the reference tensor's largest magnitude (max|y-ref| / max|ref|)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2604_00754_b200 import binding as sa
+from paper_2604_00754_b200 import workloads as wl
+from paper_2604_00754_b200.workloads import CAUSAL, LINEAR_WINDOW, SWA_ONE_SIDED, as_f64
+
+pytestmark = pytest.mark.gpu
+
+F32_ATOL = 1e-4
+BF16_REL = 2e-2
+
+
+def close(got: torch.Tensor, ref: np.ndarray, dtype, what=""):
+    g = as_f64(got)
+    err = np.abs(g - ref).max()
+    if dtype == torch.float32:
+        assert err <= F32_ATOL, "%s max-abs %.3e" % (what, err)
+    else:
+        assert err <= BF16_REL * max(np.abs(ref).max(), 1e-30), \
+            "%s rel %.3e" % (what, err / np.abs(ref).max())
+    return err
+
+
+def draw(shape_q, shape_k, dtype, seed, scale=1.0):
+    g = torch.Generator().manual_seed(seed)
+    mk = lambda s: (torch.randn(*s, generator=g) * scale).to(dtype)
+    return mk(shape_q), mk(shape_k), mk(shape_k)
+
+
+def perms(seed, layer, B, n):
+    perm, inv = sa.sa_make_perm(seed, layer, B, n)
+    return perm, inv, perm.cpu().numpy(), inv.cpu().numpy()
+
+
+# ------------------------------------------------------------------ permutation
+
+@pytest.mark.parametrize("B,n", [(1, 1), (3, 2), (2, 27), (1, 255), (2, 256), (3, 2049),
+                                 (8, 4096), (1, 32768), (2, 100000), (1, 131072)])
+def test_make_perm_bit_exact(B, n):
+    for seed, layer in [(0, 0), (0xDEADBEEFCAFEF00D, 47)]:
+        perm, inv = sa.sa_make_perm(seed, layer, B, n)
+        operm, oinv = oracle.make_perm(seed, layer, B, n)
+        assert np.array_equal(perm.cpu().numpy(), operm)
+        assert np.array_equal(inv.cpu().numpy(), oinv)
+    assert sa.sa_read_status() == 0
+
+
+def test_make_perm_sorts_tied_keys_stably():
+    # the sort itself on adversarial input is exercised through the public call only with
+    # Philox keys; equal keys cannot be forced, so check determinism run to run instead
+    a, _ = sa.sa_make_perm(5, 1, 4, 5000)
+    b, _ = sa.sa_make_perm(5, 1, 4, 5000)
+    assert torch.equal(a, b)
+
+
+# ---------------------------------------------------------------------- forward
+
+SMALL = [
+    # B, Hq, Hkv, n, d, w, flags
+    (1, 1, 1, 1, 8, 1, CAUSAL),
+    (1, 1, 1, 27, 64, 8, CAUSAL),                       # Fig. 3 shape
+    (2, 4, 2, 300, 64, 33, CAUSAL),
+    (2, 4, 2, 300, 64, 33, 0),
+    (1, 2, 1, 257, 128, 64, CAUSAL | LINEAR_WINDOW),
+    (1, 2, 2, 130, 32, 1, CAUSAL),
+    (1, 2, 2, 96, 128, 500, CAUSAL),                    # w > n: every causal key
+    (1, 2, 2, 96, 128, 96, 0),                          # w == n even: antipode excluded
+    (1, 6, 2, 511, 128, 129, CAUSAL),
+    (1, 1, 1, 700, 256, 40, 0),
+    (1, 3, 3, 64, 8, 5, LINEAR_WINDOW),
+]
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("B,Hq,Hkv,n,d,w,flags", SMALL)
+def test_sa_forward_small(B, Hq, Hkv, n, d, w, flags, dtype):
+    q, k, v = draw((B, Hq, n, d), (B, Hkv, n, d), dtype, seed=n + w)
+    perm, inv, permc, invc = perms(n, w, B, n)
+    y, lse = sa.sa_forward(q.cuda(), k.cuda(), v.cuda(), perm, inv, w, flags, want_lse=True)
+    ry, rlse = oracle.sa_forward(as_f64(q), as_f64(k), as_f64(v), permc, invc, w, flags)
+    close(y, ry, dtype, "y")
+    assert np.abs(as_f64(lse) - rlse).max() <= (1e-4 if dtype == torch.float32 else 2e-2)
+    assert sa.sa_read_status() == 0
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("B,Hq,Hkv,n,d,w,flags", [
+    (2, 4, 2, 300, 64, 33, CAUSAL | SWA_ONE_SIDED),
+    (1, 2, 1, 257, 128, 64, CAUSAL | SWA_ONE_SIDED),
+    (1, 2, 2, 96, 128, 500, CAUSAL | SWA_ONE_SIDED),
+    (1, 2, 2, 130, 64, 1, CAUSAL | SWA_ONE_SIDED),
+    (2, 4, 2, 300, 64, 33, CAUSAL),
+    (2, 4, 2, 300, 64, 33, 0),
+    (1, 1, 1, 200, 128, 31, LINEAR_WINDOW),
+])
+def test_swa_forward_small(B, Hq, Hkv, n, d, w, flags, dtype):
+    q, k, v = draw((B, Hq, n, d), (B, Hkv, n, d), dtype, seed=3 * n + w)
+    y, lse = sa.sa_swa_forward(q.cuda(), k.cuda(), v.cuda(), w, flags, want_lse=True)
+    ry, rlse = oracle.swa_forward(as_f64(q), as_f64(k), as_f64(v), w, flags)
+    close(y, ry, dtype, "y")
+    assert np.abs(as_f64(lse) - rlse).max() <= (1e-4 if dtype == torch.float32 else 2e-2)
+
+
+def test_identity_permutation_equals_swa_on_device():
+    B, Hq, Hkv, n, d, w = 1, 2, 1, 333, 64, 17
+    q, k, v = draw((B, Hq, n, d), (B, Hkv, n, d), torch.float32, seed=1)
+    ident = torch.arange(n, dtype=torch.int32, device="cuda")[None].contiguous()
+    y1 = sa.sa_forward(q.cuda(), k.cuda(), v.cuda(), ident, ident, w, CAUSAL)
+    y2 = sa.sa_swa_forward(q.cuda(), k.cuda(), v.cuda(), w, CAUSAL)
+    assert torch.equal(y1, y2)
+
+
+def test_token_major_strides():
+    # [B,n,H,d] storage viewed as [B,H,n,d]
+    B, Hq, Hkv, n, d, w = 2, 4, 2, 200, 64, 21
+    q, k, v = draw((B, Hq, n, d), (B, Hkv, n, d), torch.bfloat16, seed=9)
+    tm = lambda t: t.cuda().permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3)
+    perm, inv, permc, invc = perms(9, 0, B, n)
+    qd, kd, vd = tm(q), tm(k), tm(v)
+    assert not qd.is_contiguous()
+    y = sa.sa_forward(qd, kd, vd, perm, inv, w, CAUSAL, y=torch.empty_like(qd))
+    ry, _ = oracle.sa_forward(as_f64(q), as_f64(k), as_f64(v), permc, invc, w, CAUSAL)
+    close(y, ry, torch.bfloat16)
+
+
+def test_softmax_scale():
+    B, Hq, Hkv, n, d, w = 1, 1, 1, 100, 64, 9
+    q, k, v = draw((B, Hq, n, d), (B, Hkv, n, d), torch.float32, seed=2)
+    perm, inv, permc, invc = perms(2, 0, B, n)
+    y = sa.sa_forward(q.cuda(), k.cuda(), v.cuda(), perm, inv, w, 0, scale=0.05)
+    ry, _ = oracle.sa_forward(as_f64(q), as_f64(k), as_f64(v), permc, invc, w, 0, scale=0.05)
+    close(y, ry, torch.float32)
+
+
+def test_config_c1_full():
+    c = wl.C1
+    t = wl.draw(c)
+    perm, inv, permc, invc = perms(c.seed, 0, c.B, c.n)
+    y = sa.sa_forward(t["q"].cuda(), t["k"].cuda(), t["v"].cuda(), perm, inv, c.w, c.flags)
+    ry, _ = oracle.sa_forward(as_f64(t["q"]), as_f64(t["k"]), as_f64(t["v"]), permc, invc, c.w,
+                              c.flags)
+    close(y, ry, torch.float32, "C1")
+    assert np.array_equal(permc, oracle.make_perm(c.seed, 0, c.B, c.n)[0])
+
+
+def test_config_c2_full():
+    c = wl.C2
+    t = wl.draw(c)
+    perm, inv, permc, invc = perms(c.seed, 0, c.B, c.n)
+    operm, oinv = oracle.make_perm(c.seed, 0, c.B, c.n)
+    assert np.array_equal(permc, operm) and np.array_equal(invc, oinv)
+    y = sa.sa_forward(t["q"].cuda(), t["k"].cuda(), t["v"].cuda(), perm, inv, c.w, c.flags)
+    ry, _ = oracle.sa_forward(as_f64(t["q"]), as_f64(t["k"]), as_f64(t["v"]), operm, oinv, c.w,
+                              c.flags)
+    close(y, ry, torch.bfloat16, "C2")
+
+
+def sample_rows(c, rng, count):
+    """Random rows plus every row of the first / last 128 slots' worth of tokens."""
+    total = c.B * c.Hq * c.n
+    rows = rng.choice(total, size=count, replace=False)
+    edge = np.concatenate([np.arange(0, 128), np.arange(c.n - 128, c.n)])
+    return np.unique(np.concatenate([rows, edge, (c.Hq - 1) * c.n + edge])).astype(np.int64)
+
+
+def gated_rows_reference(c, t, permc, invc, rows):
+    q, k, v = as_f64(t["q"]), as_f64(t["k"]), as_f64(t["v"])
+    ysa, lsa = oracle.forward_rows(0, q, k, v, permc, invc, c.w, c.flags, rows)
+    ysw, lsw = oracle.forward_rows(1, q, k, v, None, None, c.w, c.flags, rows)
+    lg = t["gate_logits"].double().numpy()
+    hq = (rows // c.n) % c.Hq
+    g = 1 / (1 + np.exp(-lg))
+    return g[0, hq][:, None] * ysa + g[1, hq][:, None] * ysw, ysa, ysw, lsa, lsw
+
+
+def test_config_c3_sampled_rows():
+    c = wl.C3
+    t = wl.draw(c)
+    perm, inv, permc, invc = perms(c.seed, 0, c.B, c.n)
+    operm, oinv = oracle.make_perm(c.seed, 0, c.B, c.n)
+    assert np.array_equal(permc, operm) and np.array_equal(invc, oinv)
+    d = {k_: v_.cuda() for k_, v_ in t.items()}
+    y, y_sa, y_swa, lse_sa, lse_swa = sa.sa_swa_gated_forward(
+        d["q"], d["k"], d["v"], perm, inv, d["gate_logits"], c.w, c.flags, save_for_bwd=True)
+    y_only_sa = sa.sa_forward(d["q"], d["k"], d["v"], perm, inv, c.w, c.flags)
+    assert torch.equal(y_only_sa, y_sa)
+    rows = sample_rows(c, np.random.default_rng(0), 4096)
+    ry, rysa, rysw, rlsa, rlsw = gated_rows_reference(c, t, operm, oinv, rows)
+    flat = lambda x: x.reshape(-1, c.d)[torch.from_numpy(rows).cuda()]
+    close(flat(y), ry, torch.bfloat16, "y")
+    close(flat(y_sa), rysa, torch.bfloat16, "y_sa")
+    close(flat(y_swa), rysw, torch.bfloat16, "y_swa")
+    assert np.abs(as_f64(lse_sa.reshape(-1)[torch.from_numpy(rows).cuda()]) - rlsa).max() < 2e-2
+    assert np.abs(as_f64(lse_swa.reshape(-1)[torch.from_numpy(rows).cuda()]) - rlsw).max() < 2e-2
+    # a property that holds at any size: each output row is a convex combination of V rows
+    vmax = d["v"].float().norm(dim=-1).max()
+    assert y_sa.float().norm(dim=-1).max() <= vmax * 1.01
+    assert sa.sa_read_status() == 0
+
+
+def test_config_c4_two_layers_sampled_rows():
+    c = wl.C4
+    t = wl.draw(c)
+    d = {k_: v_.cuda() for k_, v_ in t.items()}
+    rng = np.random.default_rng(1)
+    for layer in (0, c.layers - 1):
+        perm, inv, permc, invc = perms(c.seed, layer, c.B, c.n)
+        operm, oinv = oracle.make_perm(c.seed, layer, c.B, c.n)
+        assert np.array_equal(permc, operm) and np.array_equal(invc, oinv)
+        y = sa.sa_swa_gated_forward(d["q"], d["k"], d["v"], perm, inv, d["gate_logits"], c.w,
+                                    c.flags)
+        rows = sample_rows(c, rng, 1024)
+        ry = gated_rows_reference(c, t, operm, oinv, rows)[0]
+        close(y.reshape(-1, c.d)[torch.from_numpy(rows).cuda()], ry, torch.bfloat16, "C4 y")
+    assert sa.sa_read_status() == 0
+
+
+# ------------------------------------------------------------------------ gated
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("save", [False, True])
+def test_gated_forward_small(dtype, save):
+    B, Hq, Hkv, n, d, w = 2, 4, 2, 391, 64, 50
+    flags = CAUSAL | SWA_ONE_SIDED
+    q, k, v = draw((B, Hq, n, d), (B, Hkv, n, d), dtype, seed=77)
+    lg = torch.randn(2, Hq, generator=torch.Generator().manual_seed(5))
+    perm, inv, permc, invc = perms(77, 2, B, n)
+    out = sa.sa_swa_gated_forward(q.cuda(), k.cuda(), v.cuda(), perm, inv, lg.cuda(), w, flags,
+                                  save_for_bwd=save)
+    ref = oracle.gated_forward(as_f64(q), as_f64(k), as_f64(v), permc, invc, lg.double().numpy(),
+                               w, flags)
+    if save:
+        for got, r, name in zip(out[:3], ref[:3], ("y", "y_sa", "y_swa")):
+            close(got, r, dtype, name)
+        for got, r in zip(out[3:], ref[3:]):
+            assert np.abs(as_f64(got) - r).max() <= (1e-4 if dtype == torch.float32 else 2e-2)
+    else:
+        close(out, ref[0], dtype, "y")
+
+
+# --------------------------------------------------------------------- backward
+
+def run_backward(q, k, v, dy, lg, perm, inv, w, flags):
+    qd, kd, vd, dyd = q.cuda(), k.cuda(), v.cuda(), dy.cuda()
+    if lg is None:
+        y, lse = sa.sa_forward(qd, kd, vd, perm, inv, w, flags, want_lse=True)
+        return sa.sa_backward(qd, kd, vd, perm, inv, None, y, None, lse, None, dyd, w, flags)
+    y, y_sa, y_swa, lse_sa, lse_swa = sa.sa_swa_gated_forward(qd, kd, vd, perm, inv, lg.cuda(), w,
+                                                              flags, save_for_bwd=True)
+    return sa.sa_backward(qd, kd, vd, perm, inv, lg.cuda(), y_sa, y_swa, lse_sa, lse_swa, dyd, w,
+                          flags)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("gated", [False, True])
+@pytest.mark.parametrize("B,Hq,Hkv,n,d,w,flags", [
+    (2, 4, 2, 200, 64, 21, CAUSAL | SWA_ONE_SIDED),
+    (1, 2, 2, 130, 128, 40, 0),
+    (1, 2, 1, 77, 32, 300, CAUSAL),
+    (1, 1, 1, 260, 64, 1, CAUSAL | SWA_ONE_SIDED),
+])
+def test_backward_small(B, Hq, Hkv, n, d, w, flags, gated, dtype):
+    q, k, v = draw((B, Hq, n, d), (B, Hkv, n, d), dtype, seed=n)
+    g = torch.Generator().manual_seed(n + 1)
+    dy = torch.randn(B, Hq, n, d, generator=g).to(dtype)
+    lg = torch.randn(2, Hq, generator=g) if gated else None
+    perm, inv, permc, invc = perms(n, 1, B, n)
+    dq, dk, dv, dg = run_backward(q, k, v, dy, lg, perm, inv, w, flags)
+    rdq, rdk, rdv, rdg = oracle.backward(as_f64(q), as_f64(k), as_f64(v), permc, invc,
+                                         None if lg is None else lg.double().numpy(),
+                                         as_f64(dy), w, flags)
+    if dtype == torch.float32:
+        # gradients are sums of up to band*G terms of size O(1): scale the fp32 bound
+        for got, r, name in ((dq, rdq, "dq"), (dk, rdk, "dk"), (dv, rdv, "dv")):
+            assert np.abs(as_f64(got) - r).max() <= 1e-4 * max(1.0, np.abs(r).max()), name
+        if gated:
+            assert np.abs(as_f64(dg) - rdg).max() <= 1e-4 * max(1.0, np.abs(rdg).max())
+    else:
+        close(dq, rdq, dtype, "dq")
+        close(dk, rdk, dtype, "dk")
+        close(dv, rdv, dtype, "dv")
+        if gated:
+            close(dg, rdg, dtype, "dgate")
+    assert sa.sa_read_status() == 0
+
+
+def test_config_c5_one_layer_full():
+    c = wl.C5
+    t = wl.draw(c)
+    perm, inv, permc, invc = perms(c.seed, 0, c.B, c.n)
+    dq, dk, dv, dg = run_backward(t["q"], t["k"], t["v"], t["dy"], t["gate_logits"], perm, inv,
+                                  c.w, c.flags)
+    rdq, rdk, rdv, rdg = oracle.backward(as_f64(t["q"]), as_f64(t["k"]), as_f64(t["v"]), permc,
+                                         invc, t["gate_logits"].double().numpy(),
+                                         as_f64(t["dy"]), c.w, c.flags)
+    close(dq, rdq, torch.bfloat16, "dq")
+    close(dk, rdk, torch.bfloat16, "dk")
+    close(dv, rdv, torch.bfloat16, "dv")
+    close(dg, rdg, torch.bfloat16, "dgate")
+    y = sa.sa_swa_gated_forward(t["q"].cuda(), t["k"].cuda(), t["v"].cuda(), perm, inv,
+                                t["gate_logits"].cuda(), c.w, c.flags)
+    ry = oracle.gated_forward(as_f64(t["q"]), as_f64(t["k"]), as_f64(t["v"]), permc, invc,
+                              t["gate_logits"].double().numpy(), c.w, c.flags)[0]
+    close(y, ry, torch.bfloat16, "y")
+
+
+def test_backward_is_deterministic():
+    B, Hq, Hkv, n, d, w = 1, 4, 2, 500, 64, 33
+    q, k, v = draw((B, Hq, n, d), (B, Hkv, n, d), torch.bfloat16, seed=4)
+    g = torch.Generator().manual_seed(8)
+    dy = torch.randn(B, Hq, n, d, generator=g).to(torch.bfloat16)
+    lg = torch.randn(2, Hq, generator=g)
+    perm, inv, _, _ = perms(4, 0, B, n)
+    a = run_backward(q, k, v, dy, lg, perm, inv, w, CAUSAL | SWA_ONE_SIDED)
+    b = run_backward(q, k, v, dy, lg, perm, inv, w, CAUSAL | SWA_ONE_SIDED)
+    for x, y in zip(a, b):
+        assert torch.equal(x, y)
+
+
+# --------------------------------------------------------------------- coverage
+
+@pytest.mark.parametrize("n,w,flags,L", [(2048, 32, 0, 6), (2048, 32, CAUSAL, 6), (27, 8, CAUSAL, 3),
+                                         (1000, 9, LINEAR_WINDOW, 5), (64, 200, 0, 2),
+                                         (50, 50, 0, 2)])
+def test_coverage_bit_exact(n, w, flags, L):
+    pl = [sa.sa_make_perm(31, l, 1, n) for l in range(L)]
+    perm = torch.cat([a for a, _ in pl]).contiguous()
+    inv = torch.cat([b for _, b in pl]).contiguous()
+    for src in (0, n - 1, n // 3):
+        nnz, rc, reach = sa.sa_coverage(perm, inv, w, flags, src)
+        onnz, orc, oreach = oracle.coverage(perm.cpu().numpy(), inv.cpu().numpy(), w, flags, src)
+        assert np.array_equal(nnz.cpu().numpy(), onnz)
+        assert np.array_equal(rc.cpu().numpy(), orc)
+        assert np.array_equal(reach.cpu().numpy(), oreach)
+
+
+# ----------------------------------------------------------------------- status
+
+def test_validate_perm_reports_a_non_bijection():
+    B, Hq, Hkv, n, d, w = 1, 1, 1, 64, 64, 9
+    q, k, v = draw((B, Hq, n, d), (B, Hkv, n, d), torch.float32, seed=6)
+    perm, inv, _, _ = perms(6, 0, B, n)
+    y = sa.sa_forward(q.cuda(), k.cuda(), v.cuda(), perm, inv, w, CAUSAL | wl.VALIDATE_PERM)
+    assert sa.sa_read_status() == 0
+    bad = perm.clone()
+    bad[0, 5] = bad[0, 6]                 # in range, but token repeated: not a bijection
+    sa.sa_forward(q.cuda(), k.cuda(), v.cuda(), bad, inv, w, CAUSAL | wl.VALIDATE_PERM)
+    assert sa.sa_read_status() == 5       # SA_ERR_BAD_PERM
+    assert sa.sa_read_status() == 0       # reading clears it
+    y2 = sa.sa_forward(q.cuda(), k.cuda(), v.cuda(), perm, inv, w, CAUSAL | wl.VALIDATE_PERM)
+    assert torch.equal(y, y2)
