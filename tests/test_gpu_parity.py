@@ -22,8 +22,10 @@ def close(got: torch.Tensor, ref: np.ndarray, dtype, what=""):
     if dtype == torch.float32:
         assert err <= F32_ATOL, "%s max-abs %.3e" % (what, err)
     else:
-        assert err <= BF16_REL * max(np.abs(ref).max(), 1e-30), \
-            "%s rel %.3e" % (what, err / np.abs(ref).max())
+        # 1e-5 floor: a reference that is identically zero (w = 1 gives dq = dk = 0) still
+        # meets bf16 roundings of cancelling terms
+        assert err <= BF16_REL * np.abs(ref).max() + 1e-5, \
+            "%s rel %.3e" % (what, err / max(np.abs(ref).max(), 1e-30))
     return err
 
 
