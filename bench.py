@@ -177,6 +177,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="C3")
+    ap.add_argument("--n", type=int, default=0,
+                    help="override the sequence length (profiling captures on a smaller case)")
     ap.add_argument("--no-extras", action="store_true",
                     help="skip the side measurements (SWA, backward, e2e, CPU oracle)")
     args = ap.parse_args()
@@ -184,6 +186,8 @@ def main():
 
     from paper_2604_00754_b200 import workloads as wl
     c = {k.split("_")[0]: v for k, v in wl.CONFIGS.items()}[args.workload]
+    if args.n:
+        c = c.scaled(n=args.n, name="%s_n%d" % (c.name, args.n))
     if args.impl == "reference":
         run_reference(args, c)
         return
