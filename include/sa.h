@@ -52,7 +52,8 @@ typedef enum {
   SA_ERR_WORKSPACE = 3,   /* ws_bytes smaller than sa_workspace_bytes()                  */
   SA_ERR_CUDA = 4,        /* a CUDA runtime call failed (launch error, no device)       */
   SA_ERR_BAD_PERM = 5,    /* device: perm/inv are not mutually inverse bijections       */
-  SA_ERR_TIMEOUT = 6      /* device: a bounded wait inside a kernel ran out             */
+  SA_ERR_TIMEOUT = 6,     /* device: a bounded wait inside a kernel ran out             */
+  SA_ERR_TOO_LARGE = 7    /* sa_make_perm_static: B, n need more than the built-in scratch */
 } sa_status;
 
 typedef enum { SA_F32 = 0, SA_BF16 = 1 } sa_dtype;
@@ -102,6 +103,30 @@ size_t sa_workspace_bytes(const sa_problem* p, int op);
  * perm, inv: out, int32 [B,n].  ws: scratch of sa_workspace_bytes(.., SA_OP_MAKE_PERM). */
 sa_status sa_make_perm(uint64_t seed, uint32_t layer, int32_t B, int32_t n, int32_t* perm,
                        int32_t* inv, void* ws, size_t ws_bytes, sa_stream_t stream);
+
+/* sa_make_perm for callers that cannot allocate device memory.  The paper has no counterpart:
+ * this is the same operation as sa_make_perm with the same result, bit for bit; only the home
+ * of the sort's scratch differs.  It is meant for code that runs where cudaMalloc (or a
+ * framework's caching allocator) is off limits -- a hook called while another library holds
+ * the allocator, a real-time loop that must not touch the driver's memory manager, a plug-in
+ * that is handed output buffers and nothing else -- and so cannot provide the workspace that
+ * sa_make_perm asks for.  The scratch lives inside the library image instead: a fixed array of
+ * SA_STATIC_SCRATCH_BYTES that every GPU which loads the library holds until the process exits.
+ *   - perm, inv: out, device, int32 [B,n], 16-byte aligned, owned by the caller as always.
+ *   - Limit: sa_workspace_bytes(.., SA_OP_MAKE_PERM) for (B, n) must not exceed
+ *     SA_STATIC_SCRATCH_BYTES (about 170,000 tokens in total, B*n); beyond that the call
+ *     returns SA_ERR_TOO_LARGE and launches nothing.
+ *   - The call allocates and frees nothing, and only enqueues kernels on `stream`.
+ *   - The first call on each device looks up the array's device address (one runtime query,
+ *     with that device current); make that first call before starting any stream capture.
+ *   - All calls on a device share the one array and it keeps whatever the last call left.
+ *     No part of it has to be cleared: a call writes every word before reading it.  Two
+ *     calls whose kernels may run at the same time on one GPU (different streams, or
+ *     different host threads) race on the array and give wrong permutations: keep the
+ *     calls of a device on one stream, or order them yourself. */
+#define SA_STATIC_SCRATCH_BYTES (4u << 20)
+sa_status sa_make_perm_static(uint64_t seed, uint32_t layer, int32_t B, int32_t n,
+                              int32_t* perm, int32_t* inv, sa_stream_t stream);
 
 /* SA forward (Alg. 1; Eq. 1 on the neighbourhood of Eq. 3; mask of App. B).
  * Rows of q/k/v are gathered through perm inside the kernel and rows of y are scattered

@@ -26,7 +26,7 @@ F32, BF16 = 0, 1
 EXPORTS = [
     "sa_problem_set_contiguous", "sa_workspace_bytes", "sa_make_perm", "sa_forward",
     "sa_swa_forward", "sa_swa_gated_forward", "sa_backward", "sa_coverage", "sa_read_status",
-    "sa_status_string", "sa_launch_count", "sa_set_profile_events",
+    "sa_status_string", "sa_launch_count", "sa_set_profile_events", "sa_make_perm_static",
 ]
 
 
@@ -72,6 +72,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.sa_workspace_bytes.argtypes = [pp, ctypes.c_int]
     lib.sa_workspace_bytes.restype = sz
     lib.sa_make_perm.argtypes = [u64, u32, i32, i32, vp, vp, vp, sz, vp]
+    lib.sa_make_perm_static.argtypes = [u64, u32, i32, i32, vp, vp, vp]
+    lib.sa_make_perm_static.restype = ctypes.c_int
     lib.sa_forward.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.sa_swa_forward.argtypes = [pp, vp, vp, vp, vp, vp, vp, sz, vp]
     lib.sa_swa_gated_forward.argtypes = [pp] + [vp] * 12 + [sz, vp]
@@ -177,6 +179,27 @@ def sa_make_perm(seed: int, layer: int, B: int, n: int, device="cuda", perm=None
     ws = _workspace(nbytes, perm.device, ws)
     _check(lib.sa_make_perm(int(seed) & (2 ** 64 - 1), int(layer), B, n, _ptr(perm), _ptr(inv),
                             _ptr(ws), ws.numel(), _stream()), "sa_make_perm")
+    return perm, inv
+
+
+STATIC_SCRATCH_BYTES = 4 << 20
+
+
+def sa_make_perm_static(seed: int, layer: int, B: int, n: int, perm: torch.Tensor,
+                        inv: torch.Tensor):
+    """sa_make_perm without a workspace, for callers that must not allocate.
+
+    Same permutations as sa_make_perm, bit for bit.  The sort's scratch is a fixed array
+    inside the library (STATIC_SCRATCH_BYTES per GPU), so this wrapper creates no tensor: the
+    caller hands in both outputs (int32 [B,n], CUDA).  Raises SaError (status 7) when B*n
+    needs more scratch than is built in (roughly B*n > 170,000).  Calls that may overlap on
+    one GPU race on the shared array: keep them on one stream."""
+    lib = load_library()
+    for t in (perm, inv):
+        if t.dtype != torch.int32 or tuple(t.shape) != (B, n) or not t.is_contiguous():
+            raise ValueError("perm and inv must be contiguous int32 [B,n]")
+    _check(lib.sa_make_perm_static(int(seed) & (2 ** 64 - 1), int(layer), B, n, _ptr(perm),
+                                   _ptr(inv), _stream()), "sa_make_perm_static")
     return perm, inv
 
 

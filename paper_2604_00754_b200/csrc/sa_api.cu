@@ -263,6 +263,7 @@ const char* sa_status_string(sa_status s) {
     case SA_ERR_CUDA: return "CUDA runtime error";
     case SA_ERR_BAD_PERM: return "perm/inv are not mutually inverse permutations";
     case SA_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+    case SA_ERR_TOO_LARGE: return "B*n needs more scratch than sa_make_perm_static has built in";
     default: return "unknown status";
   }
 }

@@ -159,6 +159,25 @@ __global__ void validate_perm_kernel(const int32_t* __restrict__ perm,
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+// Built-in scratch of sa_make_perm_static: part of the library image, so every GPU that
+// loads the library holds these bytes until the process exits.  In host code this name is
+// only a host-side stand-in for the symbol, never a device address: the launcher below
+// resolves the real address with cudaGetSymbolAddress and hands that to the kernels.
+static __device__ __align__(256) unsigned char g_static_scratch[SA_STATIC_SCRATCH_BYTES];
+
+// Device address of g_static_scratch on the current device, resolved once per device.
+unsigned char* static_scratch_ptr() {
+  static unsigned char* ptrs[64] = {nullptr};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  if (!ptrs[dev]) {
+    unsigned char* q = nullptr;
+    if (cudaGetSymbolAddress((void**)&q, g_static_scratch) != cudaSuccess) return nullptr;
+    ptrs[dev] = q;
+  }
+  return ptrs[dev];
+}
+
 }  // namespace
 
 size_t make_perm_ws_bytes(int B, int n) {
@@ -211,3 +230,19 @@ cudaError_t launch_validate_perm(const int32_t* perm, const int32_t* inv, int B,
 }
 
 }  // namespace sa
+
+extern "C" sa_status sa_make_perm_static(uint64_t seed, uint32_t layer, int32_t B, int32_t n,
+                                         int32_t* perm, int32_t* inv, sa_stream_t stream) {
+  using namespace sa;
+  if (B < 1 || n < 1) return SA_ERR_INVALID_ARG;
+  if (B > 32767 || n > (1 << 30)) return SA_ERR_UNSUPPORTED;
+  if (!perm || !inv || ((uintptr_t)perm & 15u) || ((uintptr_t)inv & 15u)) return SA_ERR_INVALID_ARG;
+  if (make_perm_ws_bytes(B, n) > (size_t)SA_STATIC_SCRATCH_BYTES) return SA_ERR_TOO_LARGE;
+  unsigned char* scratch = static_scratch_ptr();
+  if (!scratch) return SA_ERR_CUDA;
+  // Nothing in the scratch has to start at zero: the key, index and histogram arrays of a
+  // call are each written in full by that call before anything reads them, so whatever
+  // the previous call left behind is never seen.
+  return launch_make_perm(seed, layer, B, n, perm, inv, scratch, (cudaStream_t)stream) ==
+                 cudaSuccess ? SA_OK : SA_ERR_CUDA;
+}
