@@ -1,19 +1,22 @@
 // Fused permuted-window attention forward for sm_100a on the 5th-generation tensor cores.
 //
-// One CTA owns two 128-row query tiles that share one stream of 128-key K/V tiles:
-// two query heads of one GQA group over the same 128 slots (group size even), or two
-// adjacent slot tiles of one head (otherwise).  Rows of Q, K and V are gathered straight
-// from HBM into 128-byte-swizzled shared-memory tiles by TMA gather (four rows per copy,
-// row numbers taken from perm), so no permuted copy of any tensor exists.  S = Q K^T and
-// O += P V run as tcgen05.mma with fp32 accumulators in tensor memory; the softmax
-// (Eq. 1, with the mask of App. B applied per element) runs in registers, one thread per
-// query row, and writes P back to tensor memory as the A operand of the second product.
-// The epilogue normalises, applies the gate of Eq. 5 when asked, and scatters each row to
-// its original position.
+// A persistent grid (one CTA per SM) walks a list of work items.  One item is two 128-row
+// query tiles that share one stream of 128-key K/V tiles: two query heads of one GQA group
+// over the same 128 slots (group size even), or two adjacent slot tiles of one head
+// (otherwise).  Rows of Q, K and V are gathered straight from HBM into 128-byte-swizzled
+// shared-memory tiles by TMA gather (four rows per copy, row numbers taken from perm), so
+// no permuted copy of any tensor exists.  S = Q K^T and O += P V run as tcgen05.mma with
+// fp32 accumulators in tensor memory; the softmax (Eq. 1, with the mask of App. B applied
+// per element) runs in registers, one thread per query row, and writes P back to tensor
+// memory as the A operand of the second product.  The epilogue normalises, applies the gate
+// of Eq. 5 when asked, and scatters each row to its original position.
 //
 // Warp roles (384 threads): warp 0 TMA producer, warp 1 MMA issuer, warp 2 TMEM
 // allocator, warps 4-7 softmax/epilogue of query tile 0, warps 8-11 of query tile 1.
-// While one tile's softmax runs, the tensor core works on the other tile.
+// While one tile's softmax runs, the tensor core works on the other tile.  K and V tiles
+// travel through one ring of shared-memory slots (K0 V0 K1 V1 ...), and every barrier is
+// addressed by counters that run on across items, so the loads, products and epilogue of
+// neighbouring items overlap.
 //
 // Every mbarrier wait is bounded; on expiry the CTA records SA_ERR_TIMEOUT in the device
 // status word, stops issuing work, drains what it started and returns.
@@ -26,8 +29,6 @@ namespace {
 
 constexpr int kTile = 128;           // query rows per tile and keys per K/V tile
 constexpr int kThreads = 384;
-constexpr int kKVStages = 2;
-constexpr int kTokStages = 4;
 constexpr uint32_t kTmemCols = 512;
 constexpr long long kWaitCycles = 2000000000ll;  // about one second
 
@@ -48,6 +49,7 @@ struct TcParams {
   int pair_heads;             // 1: tiles = two heads, same slots; 0: two slot tiles, one head
   int n_tiles;                // slot tiles of 128
   int items_per_kv;           // work items per (b, hk)
+  int total_items;
   float scale2;               // softmax scale * log2(e)
   int64_t q_row_b, q_row_h, q_col_h;    // tensor-map coordinates: row = b*row_b + h*row_h + tok
   int64_t kv_row_b, kv_row_h, kv_col_h;
@@ -174,6 +176,12 @@ __device__ __forceinline__ void tmem_wait_st() {
   asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
 
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
 // ---------------------------------------------------------------------- descriptors
 
 // Shared-memory matrix descriptor, 128-byte swizzle: start address, leading and stride
@@ -264,70 +272,73 @@ __device__ __forceinline__ int actual_slot(const TcParams& p, int v) {
 
 // ------------------------------------------------------------------- shared memory
 
+// Ring sizes: kSlots K/V tile slots, kTok key-token lists.  The token list written for K
+// tile g is overwritten at tile g + kTok.  To load that tile the producer first has to win
+// ring use 2(g + kTok), i.e. see use 2(g + kTok) - kSlots freed.  If that use is V_x it is
+// freed by the completion of P V of tile x, which was issued after the softmax of x; if it
+// is K_x, by the completion of Q K^T of x, issued after the softmax of x - 1.  The softmax
+// of tile g is therefore over when x >= g (odd difference) or x - 1 >= g (even).
 template <int D>
-struct Smem {
+struct Cfg {
   static constexpr int kTileBytes = kTile * D * 2;
   static constexpr int kChunks = D / 64;          // 128-byte column blocks per row
   static constexpr int kChunkBytes = kTile * 128;
-  alignas(1024) uint8_t q[2][kTileBytes];
-  alignas(1024) uint8_t k[kKVStages][kTileBytes];
-  alignas(1024) uint8_t v[kKVStages][kTileBytes];
-  alignas(16) int32_t ktok[kTokStages][kTile];
-  alignas(8) uint64_t q_full, k_full[kKVStages], k_empty[kKVStages], v_full[kKVStages],
-      v_empty[kKVStages], tok_full[kTokStages], s_full[2], p_ready[2], o_done;
-  uint32_t tmem_base;
-  int gave_up;
+  static constexpr int kSlots = D == 128 ? 5 : 8;
+  static constexpr int kTok = D == 128 ? 4 : 8;
+  static_assert((2 * kTok - kSlots) % 2 ? (2 * kTok - kSlots >= 1) : (2 * kTok - kSlots >= 4),
+                "token ring too short for the slot ring");
+  static constexpr int kOffQ = 0;
+  static constexpr int kOffRing = 2 * kTileBytes;
+  static constexpr int kOffTok = kOffRing + kSlots * kTileBytes;
+  static constexpr int kOffBar = kOffTok + kTok * kTile * 4;
+  // mbarriers, 8 bytes each
+  static constexpr int kBarQFull = 0, kBarQEmpty = 1, kBarSlotFull = 2,
+                       kBarSlotEmpty = kBarSlotFull + kSlots, kBarTokFull = kBarSlotEmpty + kSlots,
+                       kBarSFull = kBarTokFull + kTok, kBarPReady = kBarSFull + 2,
+                       kBarODone = kBarPReady + 2, kNumBars = kBarODone + 2;
+  static constexpr int kOffMisc = kOffBar + kNumBars * 8;   // TMEM base address, gave_up flag
+  static constexpr int kBytes = kOffMisc + 16;
+  static constexpr uint32_t kColO = 256;                     // O_t at 256 + t*D; S_t at t*128
+  static_assert(kBytes <= 232448, "shared memory");
 };
 
 // ------------------------------------------------------------------------- kernel
 
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_constant__ TcParams p) {
-  extern __shared__ uint8_t smem_raw[];
-  using S = Smem<D>;
-  S& sm = *reinterpret_cast<S*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  extern __shared__ __align__(1024) uint8_t smem[];
+  using C = Cfg<D>;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (p.abort_flag && *p.abort_flag) return;  // an earlier check rejected perm/inv (uniform)
   // Once any CTA has recorded a timeout the rest of the grid leaves at once instead of
   // each waiting out its own limit.
   if (*(volatile int*)p.status == SA_ERR_TIMEOUT) return;
-
-  const int item = blockIdx.x % p.items_per_kv;
-  const int bh = blockIdx.x / p.items_per_kv;
-  const int hk = bh % p.Hkv, b = bh / p.Hkv;
-  const Geo g = make_geo(p, item, hk);
-  volatile int* gave_up = &sm.gave_up;
+  const uint32_t sbase = smem_u32(smem);
+  if (sbase & 1023u) {                        // the swizzled tiles need 1024-byte alignment
+    if (threadIdx.x == 0) atomicCAS(p.status, SA_OK, SA_ERR_CUDA);
+    return;
+  }
+  const uint32_t bar0 = sbase + C::kOffBar;
+  auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + C::kOffMisc);
+  volatile int* gave_up = reinterpret_cast<volatile int*>(smem + C::kOffMisc + 4);
 
   if (threadIdx.x == 0) {
-    sm.gave_up = 0;
-    mbar_init(smem_u32(&sm.q_full), 1);
-    for (int s = 0; s < kKVStages; ++s) {
-      mbar_init(smem_u32(&sm.k_full[s]), 1);
-      mbar_init(smem_u32(&sm.k_empty[s]), 1);
-      mbar_init(smem_u32(&sm.v_full[s]), 1);
-      mbar_init(smem_u32(&sm.v_empty[s]), 1);
-    }
-    for (int s = 0; s < kTokStages; ++s) mbar_init(smem_u32(&sm.tok_full[s]), 1);
-    for (int t = 0; t < 2; ++t) {
-      mbar_init(smem_u32(&sm.s_full[t]), 1);
-      mbar_init(smem_u32(&sm.p_ready[t]), kTile);
-    }
-    mbar_init(smem_u32(&sm.o_done), 1);
+    *gave_up = 0;
+    for (int i = 0; i < C::kNumBars; ++i)
+      mbar_init(bar(i), (i == C::kBarPReady || i == C::kBarPReady + 1) ? kTile : 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 2) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                 ::"r"(smem_u32(&sm.tmem_base)), "r"(kTmemCols) : "memory");
+                 ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
-  const uint32_t tmem = sm.tmem_base;
-  // TMEM columns: S0 [0,128) S1 [128,256) O0 [256,256+D) O1 [384,384+D); P_t overlays the
-  // first 64 columns of S_t (two bf16 per 32-bit cell).
-  const int32_t* perm = p.perm ? p.perm + (size_t)b * p.n : nullptr;
+  const uint32_t tmem = *tmem_slot;
 
   // Registers move from the producer / issuer warps to the softmax warps, which hold a
   // whole score row each.
@@ -335,124 +346,168 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
   asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
-    const int64_t kv_row0 = b * p.kv_row_b + hk * p.kv_row_h;
-    const int kv_col0 = (int)(hk * p.kv_col_h);
     bool ok = true;
-    if (lane == 0) mbar_expect_tx(smem_u32(&sm.q_full), 2 * S::kTileBytes);
-    __syncwarp();
-    for (int t = 0; t < 2; ++t) {
-      int rows[4];
-      const int64_t row0 = b * p.q_row_b + g.hq[t] * p.q_row_h;
+    uint32_t use = 0;      // ring uses so far
+    uint32_t gt = 0;       // K tiles so far
+    uint32_t it = 0;       // items so far
+    auto ring_wait = [&](uint32_t u) {
+      const uint32_t round = u / C::kSlots;
+      bool r = true;
+      if (round) r = mbar_wait(bar(C::kBarSlotEmpty + u % C::kSlots), (round - 1) & 1u, gave_up,
+                               p.status);
+      return (bool)__all_sync(0xffffffffu, r);
+    };
+    auto load_tile = [&](const CUtensorMap* tm, uint32_t dst, int col0, const int (&rows)[4],
+                         uint32_t mb) {
 #pragma unroll
-      for (int r = 0; r < 4; ++r) {
-        const int slot = min(g.q0[t] + 4 * lane + r, p.n - 1);
-        rows[r] = (int)(row0 + (perm ? perm[slot] : slot));
+      for (int c = 0; c < C::kChunks; ++c)
+        tma_gather4(dst + c * C::kChunkBytes + lane * 512, tm, col0 + 64 * c, rows[0], rows[1],
+                    rows[2], rows[3], mb);
+    };
+    for (int w_item = blockIdx.x; w_item < p.total_items && ok; w_item += gridDim.x, ++it) {
+      const int item = w_item % p.items_per_kv, bh = w_item / p.items_per_kv;
+      const int hk = bh % p.Hkv, b = bh / p.Hkv;
+      const Geo g = make_geo(p, item, hk);
+      const int32_t* perm = p.perm ? p.perm + (size_t)b * p.n : nullptr;
+      const int64_t kv_row0 = b * p.kv_row_b + hk * p.kv_row_h;
+      const int kv_col0 = (int)(hk * p.kv_col_h);
+      for (int j = 0; j < g.T && ok; ++j, ++gt) {
+        int rows[4], toks[4];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+          const int slot = actual_slot(p, g.kstart + j * kTile + 4 * lane + r);
+          toks[r] = perm ? perm[slot] : slot;
+          rows[r] = (int)(kv_row0 + toks[r]);
+        }
+        // K_j and the tokens of its keys
+        if (!(ok = ring_wait(use))) break;
+        {
+          const uint32_t mb = bar(C::kBarSlotFull + use % C::kSlots);
+          *reinterpret_cast<int4*>(smem + C::kOffTok + (gt % C::kTok) * (kTile * 4) + 16 * lane) =
+              make_int4(toks[0], toks[1], toks[2], toks[3]);
+          if (lane == 0) mbar_expect_tx(mb, C::kTileBytes);
+          __syncwarp();
+          if (lane == 0) mbar_arrive(bar(C::kBarTokFull + gt % C::kTok));
+          load_tile(&p.tm_k, sbase + C::kOffRing + (use % C::kSlots) * C::kTileBytes, kv_col0, rows,
+                    mb);
+          ++use;
+        }
+        if (j == 0) {
+          // Q of this item, once the products of the previous item no longer read it
+          if (it) ok = mbar_wait(bar(C::kBarQEmpty), (it - 1) & 1u, gave_up, p.status);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          if (lane == 0) mbar_expect_tx(bar(C::kBarQFull), 2 * C::kTileBytes);
+          __syncwarp();
+          for (int t = 0; t < 2; ++t) {
+            int qrows[4];
+            const int64_t row0 = b * p.q_row_b + g.hq[t] * p.q_row_h;
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+              const int slot = min(g.q0[t] + 4 * lane + r, p.n - 1);
+              qrows[r] = (int)(row0 + (perm ? perm[slot] : slot));
+            }
+            load_tile(&p.tm_q, sbase + C::kOffQ + t * C::kTileBytes, (int)(g.hq[t] * p.q_col_h),
+                      qrows, bar(C::kBarQFull));
+          }
+        }
+        // V_j
+        if (!(ok = ring_wait(use))) break;
+        {
+          const uint32_t mb = bar(C::kBarSlotFull + use % C::kSlots);
+          if (lane == 0) mbar_expect_tx(mb, C::kTileBytes);
+          __syncwarp();
+          load_tile(&p.tm_v, sbase + C::kOffRing + (use % C::kSlots) * C::kTileBytes, kv_col0, rows,
+                    mb);
+          ++use;
+        }
       }
-#pragma unroll
-      for (int c = 0; c < S::kChunks; ++c)
-        tma_gather4(smem_u32(&sm.q[t][c * S::kChunkBytes + lane * 512]), &p.tm_q,
-                    (int)(g.hq[t] * p.q_col_h) + 64 * c, rows[0], rows[1], rows[2], rows[3],
-                    smem_u32(&sm.q_full));
-    }
-    for (int j = 0; j < g.T && ok; ++j) {
-      const int s = j % kKVStages;
-      const uint32_t par = (uint32_t)(j / kKVStages) & 1u;
-      int rows[4], toks[4];
-#pragma unroll
-      for (int r = 0; r < 4; ++r) {
-        const int slot = actual_slot(p, g.kstart + j * kTile + 4 * lane + r);
-        toks[r] = perm ? perm[slot] : slot;
-        rows[r] = (int)(kv_row0 + toks[r]);
-      }
-      if (j >= kKVStages) ok = mbar_wait(smem_u32(&sm.k_empty[s]), par ^ 1u, gave_up, p.status);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      *reinterpret_cast<int4*>(&sm.ktok[j % kTokStages][4 * lane]) =
-          make_int4(toks[0], toks[1], toks[2], toks[3]);
-      if (lane == 0) mbar_expect_tx(smem_u32(&sm.k_full[s]), S::kTileBytes);
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&sm.tok_full[j % kTokStages]));
-#pragma unroll
-      for (int c = 0; c < S::kChunks; ++c)
-        tma_gather4(smem_u32(&sm.k[s][c * S::kChunkBytes + lane * 512]), &p.tm_k,
-                    kv_col0 + 64 * c, rows[0], rows[1], rows[2], rows[3],
-                    smem_u32(&sm.k_full[s]));
-      if (j >= kKVStages) ok = mbar_wait(smem_u32(&sm.v_empty[s]), par ^ 1u, gave_up, p.status);
-      ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
-      if (lane == 0) mbar_expect_tx(smem_u32(&sm.v_full[s]), S::kTileBytes);
-      __syncwarp();
-#pragma unroll
-      for (int c = 0; c < S::kChunks; ++c)
-        tma_gather4(smem_u32(&sm.v[s][c * S::kChunkBytes + lane * 512]), &p.tm_v,
-                    kv_col0 + 64 * c, rows[0], rows[1], rows[2], rows[3],
-                    smem_u32(&sm.v_full[s]));
     }
   } else if (warp == 1) {
     // -------------------------------------------------------------- MMA issuer
     if (lane == 0) {
       constexpr uint32_t idesc_qk = instr_desc(kTile, kTile, false);
       constexpr uint32_t idesc_pv = instr_desc(kTile, D, true);
-      bool ok = mbar_wait(smem_u32(&sm.q_full), 0, gave_up, p.status);
-      uint32_t p_par[2] = {0, 0};
-      int started[2] = {0, 0};     // P V has run at least once for this tile
-      auto issue_qk = [&](int t, int j) {
-        const int s = j % kKVStages;
-        const uint32_t qa = smem_u32(&sm.q[t][0]), ka = smem_u32(&sm.k[s][0]);
+      bool ok = true;
+      uint32_t use = 0, it = 0;
+      uint32_t p_cnt[2] = {0, 0};
+      auto slot_addr = [&](uint32_t u) {
+        return sbase + C::kOffRing + (u % C::kSlots) * C::kTileBytes;
+      };
+      auto slot_wait = [&](uint32_t u) {
+        return mbar_wait(bar(C::kBarSlotFull + u % C::kSlots), (u / C::kSlots) & 1u, gave_up,
+                         p.status);
+      };
+      auto issue_qk = [&](int t, uint32_t ka) {
+        const uint32_t qa = sbase + C::kOffQ + t * C::kTileBytes;
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off = (kk / 4) * S::kChunkBytes + (kk % 4) * 32;
+          const uint32_t off = (kk / 4) * C::kChunkBytes + (kk % 4) * 32;
           mma_ss(tmem + t * 128, smem_desc(qa + off, 16, 1024), smem_desc(ka + off, 16, 1024),
                  idesc_qk, kk > 0);
         }
-        tc_commit(smem_u32(&sm.s_full[t]));
+        tc_commit(bar(C::kBarSFull + t));
       };
-      auto active = [&](int t, int j) {
-        return g.valid[t] && j < g.T && tile_class(p, g.q0[t], g.kstart + j * kTile) != kSkip;
-      };
-      if (ok) ok = mbar_wait(smem_u32(&sm.k_full[0]), 0, gave_up, p.status);
-      if (ok) {
+      for (int w_item = blockIdx.x; w_item < p.total_items && ok; w_item += gridDim.x, ++it) {
+        const int item = w_item % p.items_per_kv, bh = w_item / p.items_per_kv;
+        const Geo g = make_geo(p, item, bh % p.Hkv);
+        auto active = [&](int t, int j) {
+          return g.valid[t] && j < g.T && tile_class(p, g.q0[t], g.kstart + j * kTile) != kSkip;
+        };
+        int last[2] = {-1, -1};   // last active K/V tile of each query tile
+        for (int t = 0; t < 2; ++t)
+          for (int j = g.T - 1; j >= 0; --j)
+            if (active(t, j)) { last[t] = j; break; }
+        int started[2] = {0, 0};
+        // ring uses of this item: K_j = use + 2j, V_j = use + 2j + 1
+        ok = mbar_wait(bar(C::kBarQFull), it & 1u, gave_up, p.status);
+        if (ok) ok = slot_wait(use);
+        if (!ok) break;
         tc_fence_after();
         for (int t = 0; t < 2; ++t)
-          if (active(t, 0)) issue_qk(t, 0);
-        tc_commit(smem_u32(&sm.k_empty[0]));
-      }
-      for (int j = 0; j < g.T && ok; ++j) {
-        const int s = j % kKVStages;
-        const uint32_t par = (uint32_t)(j / kKVStages) & 1u;
-        bool k_next_ready = false;
-        for (int t = 0; t < 2 && ok; ++t) {
-          if (active(t, j)) {
-            ok = mbar_wait(smem_u32(&sm.v_full[s]), par, gave_up, p.status);
-            if (ok) ok = mbar_wait(smem_u32(&sm.p_ready[t]), p_par[t], gave_up, p.status);
-            if (!ok) break;
-            p_par[t] ^= 1u;
-            tc_fence_after();
-            const uint32_t va = smem_u32(&sm.v[s][0]);
-#pragma unroll
-            for (int kk = 0; kk < kTile / 16; ++kk)
-              mma_ts(tmem + 256 + t * 128, tmem + t * 128 + kk * 8,
-                     smem_desc(va + kk * 2048, S::kChunkBytes, 1024), idesc_pv,
-                     (started[t] | kk) != 0);
-            started[t] = 1;
-          }
-          if (active(t, j + 1)) {
-            if (!k_next_ready) {
-              const int s1 = (j + 1) % kKVStages;
-              ok = mbar_wait(smem_u32(&sm.k_full[s1]), (uint32_t)((j + 1) / kKVStages) & 1u,
-                             gave_up, p.status);
+          if (active(t, 0)) issue_qk(t, slot_addr(use));
+        tc_commit(bar(C::kBarSlotEmpty + use % C::kSlots));
+        if (g.T == 1) tc_commit(bar(C::kBarQEmpty));
+        for (int j = 0; j < g.T && ok; ++j) {
+          const uint32_t uv = use + 2 * j + 1, uk = use + 2 * j + 2;
+          const bool have_next = j + 1 < g.T;
+          bool k_ready = false, v_ready = false;
+          for (int t = 0; t < 2 && ok; ++t) {
+            if (active(t, j)) {
+              if (!v_ready) { ok = slot_wait(uv); v_ready = true; }
+              if (ok) ok = mbar_wait(bar(C::kBarPReady + t), p_cnt[t] & 1u, gave_up, p.status);
               if (!ok) break;
+              ++p_cnt[t];
               tc_fence_after();
-              k_next_ready = true;
+              const uint32_t va = slot_addr(uv);
+#pragma unroll
+              for (int kk = 0; kk < kTile / 16; ++kk)
+                mma_ts(tmem + C::kColO + t * D, tmem + t * 128 + kk * 8,
+                       smem_desc(va + kk * 2048, C::kChunkBytes, 1024), idesc_pv,
+                       (started[t] | kk) != 0);
+              started[t] = 1;
+              if (j == last[t]) tc_commit(bar(C::kBarODone + t));
             }
-            issue_qk(t, j + 1);
+            if (have_next && active(t, j + 1)) {
+              if (!k_ready) {
+                ok = slot_wait(uk);
+                if (!ok) break;
+                tc_fence_after();
+                k_ready = true;
+              }
+              issue_qk(t, slot_addr(uk));
+            }
           }
+          if (ok && !v_ready) ok = slot_wait(uv);
+          if (ok && have_next && !k_ready) ok = slot_wait(uk);
+          if (!ok) break;
+          // the slots free when the products issued so far have finished
+          tc_commit(bar(C::kBarSlotEmpty + uv % C::kSlots));
+          if (have_next) tc_commit(bar(C::kBarSlotEmpty + uk % C::kSlots));
+          if (j + 2 == g.T) tc_commit(bar(C::kBarQEmpty));
         }
-        if (!ok) break;
-        tc_commit(smem_u32(&sm.v_empty[s]));
-        if (j + 1 < g.T) tc_commit(smem_u32(&sm.k_empty[(j + 1) % kKVStages]));
+        use += 2 * g.T;
       }
-      if (ok) tc_commit(smem_u32(&sm.o_done));
     }
     __syncwarp();
   }
@@ -463,110 +518,129 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
     const int row = threadIdx.x - 128 - t * 128;       // 0..127 == TMEM lane
     const uint32_t lane_addr = (uint32_t)(row & ~31) << 16;
     const uint32_t s_addr = tmem + lane_addr + t * 128;
-    const uint32_t o_addr = tmem + lane_addr + 256 + t * 128;
-    const int qv = g.q0[t] + row;
-    const bool row_valid = g.valid[t] && qv < p.n;
-    const int q_tok = row_valid ? (perm ? perm[qv] : qv) : 0;
-    float m = -INFINITY, l = 0.f;
-    uint32_t s_par = 0;
-    bool ok = true, started = false;
+    const uint32_t o_addr = tmem + lane_addr + C::kColO + t * D;
+    uint32_t s_cnt = 0, o_cnt = 0, gt = 0;
+    bool ok = true;
 
-    for (int j = 0; j < g.T && g.valid[t]; ++j) {
-      const int kv = g.kstart + j * kTile;
-      const int cls = tile_class(p, g.q0[t], kv);
-      if (cls == kSkip) continue;
-      ok = mbar_wait(smem_u32(&sm.tok_full[j % kTokStages]), (uint32_t)(j / kTokStages) & 1u,
-                     gave_up, p.status);
-      if (ok) ok = mbar_wait(smem_u32(&sm.s_full[t]), s_par, gave_up, p.status);
-      ok = __all_sync(0xffffffffu, ok);   // the tensor-memory loads below are warp-collective
-      if (!ok) break;
-      s_par ^= 1u;
-      tc_fence_after();
+    for (int w_item = blockIdx.x; w_item < p.total_items && ok; w_item += gridDim.x) {
+      const int item = w_item % p.items_per_kv, bh = w_item / p.items_per_kv;
+      const int hk = bh % p.Hkv, b = bh / p.Hkv;
+      const Geo g = make_geo(p, item, hk);
+      const uint32_t gt0 = gt;
+      gt += g.T;
+      if (!g.valid[t]) continue;
+      const int32_t* perm = p.perm ? p.perm + (size_t)b * p.n : nullptr;
+      const int qv = g.q0[t] + row;
+      const bool row_valid = qv < p.n;
+      const int q_tok = row_valid ? (perm ? perm[qv] : qv) : 0;
+      const int qcmp = (p.causal && !p.one_sided) ? q_tok : 0x7fffffff;
+      float m = -INFINITY, l = 0.f;
+      bool started = false;
 
-      float sv[kTile];
+      for (int j = 0; j < g.T; ++j) {
+        const int kv = g.kstart + j * kTile;
+        const int cls = tile_class(p, g.q0[t], kv);
+        if (cls == kSkip) continue;
+        const uint32_t tg = gt0 + j;
+        ok = mbar_wait(bar(C::kBarTokFull + tg % C::kTok), (tg / C::kTok) & 1u, gave_up, p.status);
+        if (ok) ok = mbar_wait(bar(C::kBarSFull + t), s_cnt & 1u, gave_up, p.status);
+        ok = __all_sync(0xffffffffu, ok);   // the tensor-memory loads below are warp-collective
+        if (!ok) break;
+        ++s_cnt;
+        tc_fence_after();
+
+        uint32_t sr[kTile];
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t raw[32];
-        tmem_ld32(s_addr + 32 * c, raw);
+        for (int c = 0; c < 4; ++c)
+          tmem_ld32(s_addr + 32 * c, reinterpret_cast<uint32_t(&)[32]>(sr[32 * c]));
         tmem_wait_ld();
+        const int32_t* ktok = reinterpret_cast<const int32_t*>(smem + C::kOffTok) +
+                              (tg % C::kTok) * kTile;
+        if (cls == kCausalOnly) {
 #pragma unroll
-        for (int x = 0; x < 32; ++x) sv[32 * c + x] = __uint_as_float(raw[x]);
-      }
-      const int32_t* ktok = sm.ktok[j % kTokStages];
-      if (cls == kCausalOnly) {
-#pragma unroll
-        for (int c = 0; c < kTile; c += 4) {
-          const int4 kt = *reinterpret_cast<const int4*>(ktok + c);
-          if (kt.x > q_tok) sv[c] = -INFINITY;
-          if (kt.y > q_tok) sv[c + 1] = -INFINITY;
-          if (kt.z > q_tok) sv[c + 2] = -INFINITY;
-          if (kt.w > q_tok) sv[c + 3] = -INFINITY;
-        }
-      } else if (cls == kEdge) {
-        const int q_slot = min(qv, p.n - 1);
-#pragma unroll
-        for (int c = 0; c < kTile; ++c) {
-          const int kvv = kv + c;
-          const int kt = ktok[c];
-          bool vis;
-          if (p.full_range) {
-            int dist = abs(q_slot - kvv);
-            if (!p.linear) dist = min(dist, p.n - dist);
-            vis = kvv < p.n && 2ll * dist < (long long)p.w && (!p.causal || kt <= q_tok);
-            if (p.one_sided) vis = kvv < p.n && kvv <= qv && qv - kvv <= p.w - 1;
-          } else if (p.one_sided) {
-            vis = kvv >= 0 && kvv <= qv && qv - kvv <= p.w - 1;
-          } else {
-            vis = abs(qv - kvv) <= p.h && (!p.linear || (kvv >= 0 && kvv < p.n)) &&
-                  (!p.causal || kt <= q_tok);
+          for (int c = 0; c < kTile; c += 4) {
+            const int4 kt = *reinterpret_cast<const int4*>(ktok + c);
+            if (kt.x > qcmp) sr[c] = 0xff800000u;
+            if (kt.y > qcmp) sr[c + 1] = 0xff800000u;
+            if (kt.z > qcmp) sr[c + 2] = 0xff800000u;
+            if (kt.w > qcmp) sr[c + 3] = 0xff800000u;
           }
-          if (!vis) sv[c] = -INFINITY;
+        } else if (cls == kEdge) {
+          // visible columns form one interval [lo, hi] of this row, cut by the token order
+          int lo, hi;
+          if (p.one_sided) { lo = p.full_range ? -kv : qv - (p.w - 1) - kv; hi = qv - kv; }
+          else if (p.full_range && !p.linear) { lo = -kv; hi = p.n - 1 - kv; }
+          else { lo = qv - p.h - kv; hi = qv + p.h - kv; }
+          if (p.linear || p.full_range || p.one_sided) {
+            lo = max(lo, -kv);
+            hi = min(hi, p.n - 1 - kv);
+          }
+          if (hi < lo) { lo = 1 << 30; hi = lo; }
+          const uint32_t span = (uint32_t)(hi - lo);
+#pragma unroll
+          for (int c = 0; c < kTile; c += 4) {
+            const int4 kt = *reinterpret_cast<const int4*>(ktok + c);
+            if ((uint32_t)(c - lo) > span || kt.x > qcmp) sr[c] = 0xff800000u;
+            if ((uint32_t)(c + 1 - lo) > span || kt.y > qcmp) sr[c + 1] = 0xff800000u;
+            if ((uint32_t)(c + 2 - lo) > span || kt.z > qcmp) sr[c + 2] = 0xff800000u;
+            if ((uint32_t)(c + 3 - lo) > span || kt.w > qcmp) sr[c + 3] = 0xff800000u;
+          }
         }
-      }
-      float mx = sv[0];
+        float mx0 = __uint_as_float(sr[0]), mx1 = __uint_as_float(sr[1]);
 #pragma unroll
-      for (int c = 1; c < kTile; ++c) mx = fmaxf(mx, sv[c]);
-      const float m_new = fmaxf(m, mx);
-      // Lazy rescaling: keep the old reference maximum while the new one is within 2^8.
-      const bool grow = (m_new - m) * p.scale2 > 8.f || (m == -INFINITY && m_new > -INFINITY);
-      if (!started) {
-        m = m_new;
-      } else if (__any_sync(0xffffffffu, grow)) {
-        const float f = grow ? exp2f((m - m_new) * p.scale2) : 1.f;
-        if (grow) { l *= f; m = m_new; }
-#pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-          uint32_t raw[32];
-          tmem_ld32(o_addr + 32 * c, raw);
-          tmem_wait_ld();
-#pragma unroll
-          for (int x = 0; x < 32; ++x) raw[x] = __float_as_uint(__uint_as_float(raw[x]) * f);
-          tmem_st32(o_addr + 32 * c, raw);
+        for (int c = 2; c < kTile; c += 4) {
+          mx0 = max3(mx0, __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]));
+          if (c + 2 < kTile)
+            mx1 = max3(mx1, __uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3]));
         }
-      }
-      started = true;
-      const float neg = (m == -INFINITY) ? 0.f : -m * p.scale2;
+        const float m_new = fmaxf(m, fmaxf(mx0, mx1));
+        // Lazy rescaling: keep the old reference maximum while the new one is within 2^8.
+        const bool grow = (m_new - m) * p.scale2 > 8.f || (m == -INFINITY && m_new > -INFINITY);
+        if (!started) {
+          m = m_new;
+        } else if (__any_sync(0xffffffffu, grow)) {
+          const float f = grow ? exp2f((m - m_new) * p.scale2) : 1.f;
+          if (grow) { l *= f; m = m_new; }
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
-        uint32_t pk[16];
+          for (int c = 0; c < D / 32; ++c) {
+            uint32_t raw[32];
+            tmem_ld32(o_addr + 32 * c, raw);
+            tmem_wait_ld();
 #pragma unroll
-        for (int x = 0; x < 16; ++x) {
-          const float p0 = exp2f(fmaf(sv[32 * c + 2 * x], p.scale2, neg));
-          const float p1 = exp2f(fmaf(sv[32 * c + 2 * x + 1], p.scale2, neg));
-          l += p0 + p1;
-          const __nv_bfloat162 h2 = __floats2bfloat162_rn(p0, p1);
-          pk[x] = *reinterpret_cast<const uint32_t*>(&h2);
+            for (int x = 0; x < 32; ++x) raw[x] = __float_as_uint(__uint_as_float(raw[x]) * f);
+            tmem_st32(o_addr + 32 * c, raw);
+          }
         }
-        tmem_st16(s_addr + 16 * c, pk);
+        started = true;
+        const float neg = (m == -INFINITY) ? 0.f : -m * p.scale2;
+        const float2 sc2 = make_float2(p.scale2, p.scale2), ng2 = make_float2(neg, neg);
+        float2 lsum = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          uint32_t pk[16];
+#pragma unroll
+          for (int x = 0; x < 16; ++x) {
+            const float2 a = __ffma2_rn(make_float2(__uint_as_float(sr[32 * c + 2 * x]),
+                                                    __uint_as_float(sr[32 * c + 2 * x + 1])),
+                                        sc2, ng2);
+            const float2 e = make_float2(exp2f(a.x), exp2f(a.y));
+            lsum = __fadd2_rn(lsum, e);
+            const __nv_bfloat162 h2 = __floats2bfloat162_rn(e.x, e.y);
+            pk[x] = *reinterpret_cast<const uint32_t*>(&h2);
+          }
+          tmem_st16(s_addr + 16 * c, pk);
+        }
+        l += lsum.x + lsum.y;
+        tmem_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar(C::kBarPReady + t));
       }
-      tmem_wait_st();
-      tc_fence_before();
-      mbar_arrive(smem_u32(&sm.p_ready[t]));
-    }
+      if (!ok) break;
 
-    if (ok && g.valid[t]) ok = mbar_wait(smem_u32(&sm.o_done), 0, gave_up, p.status);
-    ok = __all_sync(0xffffffffu, ok);
-    if (ok && g.valid[t]) {
+      ok = mbar_wait(bar(C::kBarODone + t), o_cnt & 1u, gave_up, p.status);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      ++o_cnt;
       tc_fence_after();
       const float inv_l = 1.f / l;
       float g_this = 1.f, g_other = 0.f;
@@ -626,13 +700,16 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
       }
       if (p.lse && row_valid)
         p.lse[((size_t)b * p.Hq + hq) * p.n + q_tok] = (m * p.scale2 + log2f(l)) * kLn2;
+      // the next item's first P V overwrites O: order these reads before the arrive that
+      // lets it start
+      tc_fence_before();
     }
   }
 
   // ----------------------------------------------------------------------- teardown
   tc_fence_before();
   __syncthreads();
-  if (sm.gave_up && warp == 0 && lane == 0) {
+  if (*gave_up && warp == 0 && lane == 0) {
     // Someone ran out of time: give copies that are still in flight a bounded chance to land
     // before the shared memory is released.
     const long long t0 = clock64();
@@ -707,7 +784,7 @@ bool tc_disabled() {
 }  // namespace
 
 bool tc_forward_supported(const FwdArgs& a, int dtype) {
-  if (tc_disabled() || dtype != SA_BF16 || a.d != 128) return false;
+  if (tc_disabled() || dtype != SA_BF16 || (a.d != 128 && a.d != 64)) return false;
   if (a.n < 1 || (int64_t)a.B * a.Hq * ((a.n + kTile - 1) / kTile) > 0x3fffffff) return false;
   int64_t rb, rh, ch;
   if (!row_view(a.qs, a.Hq, a.d, &rb, &rh, &ch)) return false;
@@ -744,13 +821,28 @@ cudaError_t launch_fwd_tc(const FwdArgs& a, cudaStream_t st) {
   p.items_per_kv = p.pair_heads ? p.n_tiles * (p.G / 2) : ((p.n_tiles + 1) / 2) * p.G;
   p.scale2 = a.scale * kLog2e;
   for (int i = 0; i < 3; ++i) p.qs[i] = a.qs[i];
+  p.total_items = a.B * a.Hkv * p.items_per_kv;
 
-  const size_t smem = sizeof(Smem<128>) + 1024;
-  cudaError_t e = cudaFuncSetAttribute(fwd_tc_kernel<128>,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-  if (e != cudaSuccess) return e;
-  const unsigned grid = (unsigned)((int64_t)a.B * a.Hkv * p.items_per_kv);
-  fwd_tc_kernel<128><<<grid, kThreads, smem, st>>>(p);
+  static int sm_count[64] = {0};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess || dev < 0 || dev >= 64) return e != cudaSuccess ? e : cudaErrorInvalidDevice;
+  if (!sm_count[dev]) {
+    e = cudaDeviceGetAttribute(&sm_count[dev], cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+  }
+  const unsigned grid = (unsigned)min(p.total_items, sm_count[dev]);
+  if (a.d == 128) {
+    const int smem = Cfg<128>::kBytes;
+    e = cudaFuncSetAttribute(fwd_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    fwd_tc_kernel<128><<<grid, kThreads, smem, st>>>(p);
+  } else {
+    const int smem = Cfg<64>::kBytes;
+    e = cudaFuncSetAttribute(fwd_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    fwd_tc_kernel<64><<<grid, kThreads, smem, st>>>(p);
+  }
   bump_launches();
   return cudaGetLastError();
 }
