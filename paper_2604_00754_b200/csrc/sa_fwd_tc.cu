@@ -4,15 +4,17 @@
 // query tiles that share one stream of 128-key K/V tiles: two query heads of one GQA group
 // over the same 128 slots (group size even), or two adjacent slot tiles of one head
 // (otherwise).  Rows of Q, K and V are gathered straight from HBM into 128-byte-swizzled
-// shared-memory tiles by TMA gather (four rows per copy, row numbers taken from perm), so
-// no permuted copy of any tensor exists.  S = Q K^T and O += P V run as tcgen05.mma with
+// shared-memory tiles with 16-byte cp.async copies (row numbers taken from perm, the swizzle
+// applied in the destination address), so no permuted copy of any tensor exists.  (TMA row
+// gather, four rows per copy, measured about 70 cycles per copy per SM on this part, a
+// quarter of what the tensor core consumes; the cp.async path is not issue-bound.)  S = Q K^T and O += P V run as tcgen05.mma with
 // fp32 accumulators in tensor memory; the softmax (Eq. 1, with the mask of App. B applied
 // per element) runs in registers, one thread per query row, and writes P back to tensor
 // memory as the A operand of the second product.  The epilogue normalises, applies the gate
 // of Eq. 5 when asked, and scatters each row to its original position.
 //
-// Warp roles (384 threads): warp 0 TMA producer, warp 1 MMA issuer, warp 2 TMEM
-// allocator, warps 4-7 softmax/epilogue of query tile 0, warps 8-11 of query tile 1.
+// Warp roles (384 threads): warp 0 MMA issuer and TMEM allocator, warps 1-3 gather
+// producers, warps 4-7 softmax/epilogue of query tile 0, warps 8-11 of query tile 1.
 // While one tile's softmax runs, the tensor core works on the other tile.  K and V tiles
 // travel through one ring of shared-memory slots (K0 V0 K1 V1 ...), and every barrier is
 // addressed by counters that run on across items, so the loads, products and epilogue of
@@ -20,8 +22,6 @@
 //
 // Every mbarrier wait is bounded; on expiry the CTA records SA_ERR_TIMEOUT in the device
 // status word, stops issuing work, drains what it started and returns.
-#include <cuda.h>
-
 #include "sa_fwd_tc.cuh"
 
 namespace sa {
@@ -29,13 +29,14 @@ namespace {
 
 constexpr int kTile = 128;           // query rows per tile and keys per K/V tile
 constexpr int kThreads = 384;
+constexpr int kProducers = 96;       // threads of the three gather warps
 constexpr uint32_t kTmemCols = 512;
 constexpr long long kWaitCycles = 2000000000ll;  // about one second
 
 enum TileClass { kSkip = 0, kFull = 1, kCausalOnly = 2, kEdge = 3 };
 
 struct TcParams {
-  CUtensorMap tm_q, tm_k, tm_v;
+  const void *q, *k, *v;
   const int32_t* perm;        // null for the SWA branch
   void* y;
   void* y_branch;
@@ -51,9 +52,8 @@ struct TcParams {
   int items_per_kv;           // work items per (b, hk)
   int total_items;
   float scale2;               // softmax scale * log2(e)
-  int64_t q_row_b, q_row_h, q_col_h;    // tensor-map coordinates: row = b*row_b + h*row_h + tok
-  int64_t kv_row_b, kv_row_h, kv_col_h;
-  int64_t qs[3];              // element strides of y / y_branch / y_other
+  int64_t qs[3];              // element strides of q / y / y_branch / y_other: batch, head, token
+  int64_t ks[3];              // element strides of k / v
 };
 
 // ----------------------------------------------------------------------------- PTX
@@ -66,10 +66,6 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
-               : "memory");
 }
 __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -97,17 +93,6 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       return false;
     }
   }
-}
-
-// Four rows of 64 bf16 (128 bytes) each, rows r0..r3 of the 2-D tensor, into 512 bytes of
-// 128-byte-swizzled shared memory.
-__device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap* tm, int col, int r0,
-                                            int r1, int r2, int r3, uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes"
-      " [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
-      ::"r"(dst), "l"(tm), "r"(col), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(bar)
-      : "memory");
 }
 
 __device__ __forceinline__ void tc_fence_before() {
@@ -281,16 +266,16 @@ __device__ __forceinline__ int actual_slot(const TcParams& p, int v) {
 template <int D>
 struct Cfg {
   static constexpr int kTileBytes = kTile * D * 2;
-  static constexpr int kChunks = D / 64;          // 128-byte column blocks per row
   static constexpr int kChunkBytes = kTile * 128;
   static constexpr int kSlots = D == 128 ? 5 : 8;
-  static constexpr int kTok = D == 128 ? 4 : 8;
+  static constexpr int kTok = D == 128 ? 3 : 8;
   static_assert((2 * kTok - kSlots) % 2 ? (2 * kTok - kSlots >= 1) : (2 * kTok - kSlots >= 4),
                 "token ring too short for the slot ring");
   static constexpr int kOffQ = 0;
   static constexpr int kOffRing = 2 * kTileBytes;
   static constexpr int kOffTok = kOffRing + kSlots * kTileBytes;
-  static constexpr int kOffBar = kOffTok + kTok * kTile * 4;
+  static constexpr int kOffQTok = kOffTok + kTok * kTile * 4;   // tokens of the two query tiles
+  static constexpr int kOffBar = kOffQTok + 2 * kTile * 4;
   // mbarriers, 8 bytes each
   static constexpr int kBarQFull = 0, kBarQEmpty = 1, kBarSlotFull = 2,
                        kBarSlotEmpty = kBarSlotFull + kSlots, kBarTokFull = kBarSlotEmpty + kSlots,
@@ -327,10 +312,12 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
   if (threadIdx.x == 0) {
     *gave_up = 0;
     for (int i = 0; i < C::kNumBars; ++i)
-      mbar_init(bar(i), (i == C::kBarPReady || i == C::kBarPReady + 1) ? kTile : 1);
+      mbar_init(bar(i), (i == C::kBarPReady || i == C::kBarPReady + 1) ? kTile
+                        : (i == C::kBarQFull || (i >= C::kBarSlotFull && i < C::kBarSlotEmpty))
+                            ? kProducers : 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 2) {
+  if (warp == 0) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                  ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -344,87 +331,143 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
   // whole score row each.
   if (warp < 4) {
   asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
-  if (warp == 0) {
-    // ------------------------------------------------------------ TMA producer
-    bool ok = true;
-    uint32_t use = 0;      // ring uses so far
-    uint32_t gt = 0;       // K tiles so far
-    uint32_t it = 0;       // items so far
-    auto ring_wait = [&](uint32_t u) {
-      const uint32_t round = u / C::kSlots;
-      bool r = true;
-      if (round) r = mbar_wait(bar(C::kBarSlotEmpty + u % C::kSlots), (round - 1) & 1u, gave_up,
-                               p.status);
-      return (bool)__all_sync(0xffffffffu, r);
+  if (warp >= 1) {
+    // ---------------------------------------------------- gather producers (warps 1-3)
+    // Each 16-byte piece of a row goes from global memory to its swizzled place in shared
+    // memory with cp.async; one warp instruction moves kRpi whole rows.  A thread signals a
+    // tile two tiles after issuing it: by then its copies have landed (wait_group), it
+    // publishes them to the tensor core's proxy (fence.proxy.async) and arrives on the
+    // tile's barrier, so the issue of later tiles overlaps the latency of earlier ones.
+    constexpr int kCpr = D / 8;            // 16-byte pieces per row
+    constexpr int kRpi = 32 / kCpr;        // rows per warp instruction
+    const int ptid = threadIdx.x - 32;     // 0..95
+    const int sub = lane / kCpr, chunk = lane % kCpr;
+    const uint32_t dst_lane = (uint32_t)(chunk >> 3) * C::kChunkBytes;
+    const __nv_bfloat16* qg = (const __nv_bfloat16*)p.q;
+    const __nv_bfloat16* kg = (const __nv_bfloat16*)p.k;
+    const __nv_bfloat16* vg = (const __nv_bfloat16*)p.v;
+    int32_t* const ktok_base = reinterpret_cast<int32_t*>(smem + C::kOffTok);
+    int32_t* const qtok = reinterpret_cast<int32_t*>(smem + C::kOffQTok);
+    uint32_t use = 0, gt = 0, it = 0;
+    int npend = 0;
+    uint32_t pend0 = 0, pend1 = 0;       // barriers of the tiles issued but not yet signalled
+
+    auto flush = [&]() {
+      if (npend) {
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        mbar_arrive(pend0);
+        if (npend == 2) mbar_arrive(pend1);
+        npend = 0;
+      }
     };
-    auto load_tile = [&](const CUtensorMap* tm, uint32_t dst, int col0, const int (&rows)[4],
-                         uint32_t mb) {
-#pragma unroll
-      for (int c = 0; c < C::kChunks; ++c)
-        tma_gather4(dst + c * C::kChunkBytes + lane * 512, tm, col0 + 64 * c, rows[0], rows[1],
-                    rows[2], rows[3], mb);
+    auto push = [&](uint32_t mb) {
+      asm volatile("cp.async.commit_group;" ::: "memory");
+      if (npend == 2) {
+        asm volatile("cp.async.wait_group 2;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        mbar_arrive(pend0);
+        pend0 = pend1;
+        pend1 = mb;
+      } else if (npend == 1) {
+        pend1 = mb;
+        npend = 2;
+      } else {
+        pend0 = mb;
+        npend = 1;
+      }
     };
-    for (int w_item = blockIdx.x; w_item < p.total_items && ok; w_item += gridDim.x, ++it) {
+    // Before blocking on a barrier that the consumers complete, hand over everything issued.
+    auto wait_free = [&](uint32_t mb, uint32_t parity) {
+      if (!mbar_try(mb, parity)) {
+        flush();
+        mbar_wait(mb, parity, gave_up, p.status);   // a failure sets *gave_up
+      }
+    };
+    auto gather = [&](const __nv_bfloat16* base, int64_t tok_stride, const int32_t* toks,
+                      uint32_t dst_tile) {
+#pragma unroll 4
+      for (int grp = warp - 1; grp < kTile / kRpi; grp += 3) {
+        const int r = grp * kRpi + sub;
+        const __nv_bfloat16* src = base + (int64_t)toks[r] * tok_stride + chunk * 8;
+        const uint32_t dst = dst_tile + dst_lane + r * 128 + (((chunk & 7) ^ (r & 7)) << 4);
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+      }
+    };
+    // Barrier over the three producer warps that also agrees on whether anyone in the CTA
+    // has given up: every producer thread leaves the loops at the same point.
+    auto group_sync_stop = [&]() {
+      uint32_t any;
+      asm volatile(
+          "{\n\t.reg .pred p, q;\n\t"
+          "setp.ne.u32 q, %1, 0;\n\t"
+          "bar.red.or.pred p, 1, 96, q;\n\t"
+          "selp.u32 %0, 1, 0, p;\n\t}"
+          : "=r"(any)
+          : "r"((uint32_t)*gave_up)
+          : "memory");
+      return any != 0;
+    };
+
+    bool live = true;
+    for (int w_item = blockIdx.x; w_item < p.total_items && live; w_item += gridDim.x, ++it) {
       const int item = w_item % p.items_per_kv, bh = w_item / p.items_per_kv;
       const int hk = bh % p.Hkv, b = bh / p.Hkv;
       const Geo g = make_geo(p, item, hk);
       const int32_t* perm = p.perm ? p.perm + (size_t)b * p.n : nullptr;
-      const int64_t kv_row0 = b * p.kv_row_b + hk * p.kv_row_h;
-      const int kv_col0 = (int)(hk * p.kv_col_h);
-      for (int j = 0; j < g.T && ok; ++j, ++gt) {
-        int rows[4], toks[4];
-#pragma unroll
-        for (int r = 0; r < 4; ++r) {
-          const int slot = actual_slot(p, g.kstart + j * kTile + 4 * lane + r);
-          toks[r] = perm ? perm[slot] : slot;
-          rows[r] = (int)(kv_row0 + toks[r]);
-        }
-        // K_j and the tokens of its keys
-        if (!(ok = ring_wait(use))) break;
-        {
-          const uint32_t mb = bar(C::kBarSlotFull + use % C::kSlots);
-          *reinterpret_cast<int4*>(smem + C::kOffTok + (gt % C::kTok) * (kTile * 4) + 16 * lane) =
-              make_int4(toks[0], toks[1], toks[2], toks[3]);
-          if (lane == 0) mbar_expect_tx(mb, C::kTileBytes);
-          __syncwarp();
-          if (lane == 0) mbar_arrive(bar(C::kBarTokFull + gt % C::kTok));
-          load_tile(&p.tm_k, sbase + C::kOffRing + (use % C::kSlots) * C::kTileBytes, kv_col0, rows,
-                    mb);
-          ++use;
+      const __nv_bfloat16* kb = kg + b * p.ks[0] + hk * p.ks[1];
+      const __nv_bfloat16* vb = vg + b * p.ks[0] + hk * p.ks[1];
+      auto key_tok = [&](int j, int r) {
+        const int slot = actual_slot(p, g.kstart + j * kTile + r);
+        return perm ? perm[slot] : slot;
+      };
+      auto q_tok = [&](int x) {        // x in 0..255: tile x/128, row x%128
+        const int slot = min(g.q0[x >> 7] + (x & 127), p.n - 1);
+        return perm ? perm[slot] : slot;
+      };
+      // tokens are fetched one tile ahead of their use
+      int tk0 = key_tok(0, ptid), tk1 = ptid < 32 ? key_tok(0, ptid + 96) : 0;
+      const int tq0 = q_tok(ptid), tq1 = q_tok(ptid + 96), tq2 = ptid < 64 ? q_tok(ptid + 192) : 0;
+      for (int j = 0; j < g.T; ++j, ++gt) {
+        // ---- K_j and the tokens of its keys
+        if (use >= (uint32_t)C::kSlots)
+          wait_free(bar(C::kBarSlotEmpty + use % C::kSlots), (use / C::kSlots - 1) & 1u);
+        int32_t* ktok = ktok_base + (gt % C::kTok) * kTile;
+        ktok[ptid] = tk0;
+        if (ptid < 32) ktok[ptid + 96] = tk1;
+        if (group_sync_stop()) { live = false; break; }
+        if (ptid == 0) mbar_arrive(bar(C::kBarTokFull + gt % C::kTok));
+        gather(kb, p.ks[2], ktok, sbase + C::kOffRing + (use % C::kSlots) * C::kTileBytes);
+        push(bar(C::kBarSlotFull + use % C::kSlots));
+        ++use;
+        if (j + 1 < g.T) {
+          tk0 = key_tok(j + 1, ptid);
+          if (ptid < 32) tk1 = key_tok(j + 1, ptid + 96);
         }
         if (j == 0) {
-          // Q of this item, once the products of the previous item no longer read it
-          if (it) ok = mbar_wait(bar(C::kBarQEmpty), (it - 1) & 1u, gave_up, p.status);
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) break;
-          if (lane == 0) mbar_expect_tx(bar(C::kBarQFull), 2 * C::kTileBytes);
-          __syncwarp();
-          for (int t = 0; t < 2; ++t) {
-            int qrows[4];
-            const int64_t row0 = b * p.q_row_b + g.hq[t] * p.q_row_h;
-#pragma unroll
-            for (int r = 0; r < 4; ++r) {
-              const int slot = min(g.q0[t] + 4 * lane + r, p.n - 1);
-              qrows[r] = (int)(row0 + (perm ? perm[slot] : slot));
-            }
-            load_tile(&p.tm_q, sbase + C::kOffQ + t * C::kTileBytes, (int)(g.hq[t] * p.q_col_h),
-                      qrows, bar(C::kBarQFull));
-          }
+          // ---- Q of this item, once the products of the previous item no longer read it
+          if (it) wait_free(bar(C::kBarQEmpty), (it - 1) & 1u);
+          qtok[ptid] = tq0;
+          qtok[ptid + 96] = tq1;
+          if (ptid < 64) qtok[ptid + 192] = tq2;
+          if (group_sync_stop()) { live = false; break; }
+          for (int t = 0; t < 2; ++t)
+            gather(qg + b * p.qs[0] + g.hq[t] * p.qs[1], p.qs[2], qtok + t * kTile,
+                   sbase + C::kOffQ + t * C::kTileBytes);
+          push(bar(C::kBarQFull));
         }
-        // V_j
-        if (!(ok = ring_wait(use))) break;
-        {
-          const uint32_t mb = bar(C::kBarSlotFull + use % C::kSlots);
-          if (lane == 0) mbar_expect_tx(mb, C::kTileBytes);
-          __syncwarp();
-          load_tile(&p.tm_v, sbase + C::kOffRing + (use % C::kSlots) * C::kTileBytes, kv_col0, rows,
-                    mb);
-          ++use;
-        }
+        // ---- V_j
+        if (use >= (uint32_t)C::kSlots)
+          wait_free(bar(C::kBarSlotEmpty + use % C::kSlots), (use / C::kSlots - 1) & 1u);
+        if (group_sync_stop()) { live = false; break; }
+        gather(vb, p.ks[2], ktok, sbase + C::kOffRing + (use % C::kSlots) * C::kTileBytes);
+        push(bar(C::kBarSlotFull + use % C::kSlots));
+        ++use;
       }
     }
-  } else if (warp == 1) {
-    // -------------------------------------------------------------- MMA issuer
+    flush();
+  } else {
+    // -------------------------------------------------------------- MMA issuer (warp 0)
     if (lane == 0) {
       constexpr uint32_t idesc_qk = instr_desc(kTile, kTile, false);
       constexpr uint32_t idesc_pv = instr_desc(kTile, D, true);
@@ -709,13 +752,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
   // ----------------------------------------------------------------------- teardown
   tc_fence_before();
   __syncthreads();
-  if (*gave_up && warp == 0 && lane == 0) {
-    // Someone ran out of time: give copies that are still in flight a bounded chance to land
-    // before the shared memory is released.
-    const long long t0 = clock64();
-    while (clock64() - t0 < 2000000ll) {}
-  }
-  if (warp == 2) {
+  if (warp == 0) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols)
                  : "memory");
@@ -723,54 +760,6 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
 }
 
 // ---------------------------------------------------------------------------- host
-
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
-                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
-                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
-    void* ptr = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) ==
-            cudaSuccess && qres == cudaDriverEntryPointSuccess)
-      fn = (EncodeTiledFn)ptr;
-  }
-  return fn;
-}
-
-// Coordinates of row (b, h, tok) in a 2-D view [rows, token_stride] of a tensor with element
-// strides s[0..2]; false when the layout cannot be viewed that way.
-bool row_view(const int64_t s[3], int H, int d, int64_t* row_b, int64_t* row_h, int64_t* col_h) {
-  const int64_t ts = s[2];
-  if (ts < d || s[0] % ts != 0) return false;
-  *row_b = s[0] / ts;
-  if (s[1] % ts == 0) {
-    *row_h = s[1] / ts;
-    *col_h = 0;
-  } else {
-    if (s[1] * (H - 1) + d > ts) return false;
-    *row_h = 0;
-    *col_h = s[1];
-  }
-  return true;
-}
-
-bool make_map(CUtensorMap* tm, const void* base, int64_t ts, int64_t rows) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn || rows <= 0 || rows > 0x7fffffffll) return false;
-  const cuuint64_t dims[2] = {(cuuint64_t)ts, (cuuint64_t)rows};
-  const cuuint64_t strides[1] = {(cuuint64_t)ts * 2};
-  const cuuint32_t box[2] = {64, 1};
-  const cuuint32_t estr[2] = {1, 1};
-  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
-            estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
 
 bool tc_disabled() {
   static int v = -1;
@@ -786,25 +775,12 @@ bool tc_disabled() {
 bool tc_forward_supported(const FwdArgs& a, int dtype) {
   if (tc_disabled() || dtype != SA_BF16 || (a.d != 128 && a.d != 64)) return false;
   if (a.n < 1 || (int64_t)a.B * a.Hq * ((a.n + kTile - 1) / kTile) > 0x3fffffff) return false;
-  int64_t rb, rh, ch;
-  if (!row_view(a.qs, a.Hq, a.d, &rb, &rh, &ch)) return false;
-  if (!row_view(a.ks, a.Hkv, a.d, &rb, &rh, &ch)) return false;
-  if (a.qs[2] > (1 << 20) || a.ks[2] > (1 << 20)) return false;
-  return encode_fn() != nullptr;
+  return true;
 }
 
 cudaError_t launch_fwd_tc(const FwdArgs& a, cudaStream_t st) {
   TcParams p{};
-  int64_t rb, rh, ch;
-  row_view(a.qs, a.Hq, a.d, &rb, &rh, &ch);
-  p.q_row_b = rb; p.q_row_h = rh; p.q_col_h = ch;
-  const int64_t q_rows = (a.B - 1) * rb + (a.Hq - 1) * rh + a.n;
-  row_view(a.ks, a.Hkv, a.d, &rb, &rh, &ch);
-  p.kv_row_b = rb; p.kv_row_h = rh; p.kv_col_h = ch;
-  const int64_t kv_rows = (a.B - 1) * rb + (a.Hkv - 1) * rh + a.n;
-  if (!make_map(&p.tm_q, a.q, a.qs[2], q_rows) || !make_map(&p.tm_k, a.k, a.ks[2], kv_rows) ||
-      !make_map(&p.tm_v, a.v, a.ks[2], kv_rows))
-    return cudaErrorInvalidValue;
+  p.q = a.q; p.k = a.k; p.v = a.v;
   p.perm = a.swa ? nullptr : a.perm;
   p.y = a.y; p.y_branch = a.y_branch; p.y_other = a.y_other; p.lse = a.lse;
   p.gate_logits = a.gate_logits;
@@ -820,7 +796,7 @@ cudaError_t launch_fwd_tc(const FwdArgs& a, cudaStream_t st) {
   p.n_tiles = (a.n + kTile - 1) / kTile;
   p.items_per_kv = p.pair_heads ? p.n_tiles * (p.G / 2) : ((p.n_tiles + 1) / 2) * p.G;
   p.scale2 = a.scale * kLog2e;
-  for (int i = 0; i < 3; ++i) p.qs[i] = a.qs[i];
+  for (int i = 0; i < 3; ++i) { p.qs[i] = a.qs[i]; p.ks[i] = a.ks[i]; }
   p.total_items = a.B * a.Hkv * p.items_per_kv;
 
   static int sm_count[64] = {0};
