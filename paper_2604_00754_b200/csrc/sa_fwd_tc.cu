@@ -95,6 +95,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
 }
 
+// Orders shared-memory writes made through the generic proxy (cp.async) that this thread
+// has observed before its later tensor-core reads of the same memory.
+__device__ __forceinline__ void fence_proxy_async() {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+}
 __device__ __forceinline__ void tc_fence_before() {
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
 }
@@ -169,14 +174,15 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
 
 // ---------------------------------------------------------------------- descriptors
 
-// Shared-memory matrix descriptor, 128-byte swizzle: start address, leading and stride
-// byte offsets in 16-byte units, descriptor version 1 (sm_100), layout type 2.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
-                                              uint32_t sbo_bytes) {
-  return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) |
-         ((uint64_t)(sbo_bytes >> 4) << 32) | (1ull << 46) | (2ull << 61);
+__device__ __forceinline__ uint64_t desc64(uint32_t lo, uint32_t hi) {
+  uint64_t d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
+  return d;
 }
 
+// Shared-memory matrix descriptor (128-byte swizzle): bits 0-13 start address, 16-29 leading
+// byte offset, 32-45 stride byte offset (all in 16-byte units), bit 46 descriptor version 1
+// (sm_100), bits 61-63 layout type 2.  The issuer assembles it from two prepared words.
 // Instruction descriptor, kind::f16: fp32 accumulator, bf16 A and B, A K-major.
 __host__ __device__ constexpr uint32_t instr_desc(int m, int n, bool b_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) |
@@ -334,10 +340,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
   if (warp >= 1) {
     // ---------------------------------------------------- gather producers (warps 1-3)
     // Each 16-byte piece of a row goes from global memory to its swizzled place in shared
-    // memory with cp.async; one warp instruction moves kRpi whole rows.  A thread signals a
-    // tile two tiles after issuing it: by then its copies have landed (wait_group), it
-    // publishes them to the tensor core's proxy (fence.proxy.async) and arrives on the
-    // tile's barrier, so the issue of later tiles overlaps the latency of earlier ones.
+    // memory with cp.async; one warp instruction moves kRpi whole rows.
     constexpr int kCpr = D / 8;            // 16-byte pieces per row
     constexpr int kRpi = 32 / kCpr;        // rows per warp instruction
     const int ptid = threadIdx.x - 32;     // 0..95
@@ -349,40 +352,15 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
     int32_t* const ktok_base = reinterpret_cast<int32_t*>(smem + C::kOffTok);
     int32_t* const qtok = reinterpret_cast<int32_t*>(smem + C::kOffQTok);
     uint32_t use = 0, gt = 0, it = 0;
-    int npend = 0;
-    uint32_t pend0 = 0, pend1 = 0;       // barriers of the tiles issued but not yet signalled
-
-    auto flush = [&]() {
-      if (npend) {
-        asm volatile("cp.async.wait_group 0;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        mbar_arrive(pend0);
-        if (npend == 2) mbar_arrive(pend1);
-        npend = 0;
-      }
+    // A tile's barrier counts one arrival per producer thread, triggered by the hardware
+    // when that thread's copies have landed (cp.async.mbarrier.arrive.noinc), so issuing
+    // never waits for data.  The consumer publishes the data to the tensor core's proxy
+    // (fence.proxy.async) after its wait.
+    auto signal = [&](uint32_t mb) {
+      asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(mb) : "memory");
     };
-    auto push = [&](uint32_t mb) {
-      asm volatile("cp.async.commit_group;" ::: "memory");
-      if (npend == 2) {
-        asm volatile("cp.async.wait_group 2;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        mbar_arrive(pend0);
-        pend0 = pend1;
-        pend1 = mb;
-      } else if (npend == 1) {
-        pend1 = mb;
-        npend = 2;
-      } else {
-        pend0 = mb;
-        npend = 1;
-      }
-    };
-    // Before blocking on a barrier that the consumers complete, hand over everything issued.
     auto wait_free = [&](uint32_t mb, uint32_t parity) {
-      if (!mbar_try(mb, parity)) {
-        flush();
-        mbar_wait(mb, parity, gave_up, p.status);   // a failure sets *gave_up
-      }
+      mbar_wait(mb, parity, gave_up, p.status);     // a failure sets *gave_up
     };
     auto gather = [&](const __nv_bfloat16* base, int64_t tok_stride, const int32_t* toks,
                       uint32_t dst_tile) {
@@ -438,7 +416,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
         if (group_sync_stop()) { live = false; break; }
         if (ptid == 0) mbar_arrive(bar(C::kBarTokFull + gt % C::kTok));
         gather(kb, p.ks[2], ktok, sbase + C::kOffRing + (use % C::kSlots) * C::kTileBytes);
-        push(bar(C::kBarSlotFull + use % C::kSlots));
+        signal(bar(C::kBarSlotFull + use % C::kSlots));
         ++use;
         if (j + 1 < g.T) {
           tk0 = key_tok(j + 1, ptid);
@@ -454,61 +432,78 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
           for (int t = 0; t < 2; ++t)
             gather(qg + b * p.qs[0] + g.hq[t] * p.qs[1], p.qs[2], qtok + t * kTile,
                    sbase + C::kOffQ + t * C::kTileBytes);
-          push(bar(C::kBarQFull));
+          signal(bar(C::kBarQFull));
         }
         // ---- V_j
         if (use >= (uint32_t)C::kSlots)
           wait_free(bar(C::kBarSlotEmpty + use % C::kSlots), (use / C::kSlots - 1) & 1u);
         if (group_sync_stop()) { live = false; break; }
         gather(vb, p.ks[2], ktok, sbase + C::kOffRing + (use % C::kSlots) * C::kTileBytes);
-        push(bar(C::kBarSlotFull + use % C::kSlots));
+        signal(bar(C::kBarSlotFull + use % C::kSlots));
         ++use;
       }
     }
-    flush();
+    asm volatile("cp.async.wait_all;" ::: "memory");   // nothing in flight when the CTA leaves
   } else {
     // -------------------------------------------------------------- MMA issuer (warp 0)
+    // One thread feeds the tensor core, so every instruction between two tcgen05.mma counts:
+    // the descriptors are built from words prepared outside the loops and the K steps are
+    // fully unrolled with immediate offsets.
     if (lane == 0) {
       constexpr uint32_t idesc_qk = instr_desc(kTile, kTile, false);
       constexpr uint32_t idesc_pv = instr_desc(kTile, D, true);
+      // shared-memory descriptor words (128-byte swizzle, 1024 bytes between 8-row groups)
+      constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+      constexpr uint32_t kLoK = (16u >> 4) << 16;                          // K-major operands
+      constexpr uint32_t kLoV = ((uint32_t)C::kChunkBytes >> 4) << 16;     // V: next 64 columns
+      const uint32_t q_lo[2] = {((sbase + C::kOffQ) >> 4) | kLoK,
+                                ((sbase + C::kOffQ + C::kTileBytes) >> 4) | kLoK};
+      const uint32_t ring_lo = (sbase + C::kOffRing) >> 4;
       bool ok = true;
       uint32_t use = 0, it = 0;
       uint32_t p_cnt[2] = {0, 0};
-      auto slot_addr = [&](uint32_t u) {
-        return sbase + C::kOffRing + (u % C::kSlots) * C::kTileBytes;
-      };
+      auto slot_lo = [&](uint32_t u) { return ring_lo + (u % C::kSlots) * (C::kTileBytes >> 4); };
       auto slot_wait = [&](uint32_t u) {
         return mbar_wait(bar(C::kBarSlotFull + u % C::kSlots), (u / C::kSlots) & 1u, gave_up,
                          p.status);
       };
-      auto issue_qk = [&](int t, uint32_t ka) {
-        const uint32_t qa = sbase + C::kOffQ + t * C::kTileBytes;
+      auto issue_qk = [&](int t, uint32_t k_lo) {
+        const uint32_t ql = q_lo[t], kl = k_lo | kLoK, d = tmem + t * 128;
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off = (kk / 4) * C::kChunkBytes + (kk % 4) * 32;
-          mma_ss(tmem + t * 128, smem_desc(qa + off, 16, 1024), smem_desc(ka + off, 16, 1024),
-                 idesc_qk, kk > 0);
+          const uint32_t off = (kk / 4) * (C::kChunkBytes >> 4) + (kk % 4) * 2;
+          mma_ss(d, desc64(ql + off, kDescHi), desc64(kl + off, kDescHi), idesc_qk, kk > 0);
         }
         tc_commit(bar(C::kBarSFull + t));
+      };
+      auto issue_pv = [&](int t, uint32_t v_lo, uint32_t acc0) {
+        const uint32_t vl = v_lo | kLoV, d = tmem + C::kColO + t * D, a = tmem + t * 128;
+#pragma unroll
+        for (int kk = 0; kk < kTile / 16; ++kk)
+          mma_ts(d, a + kk * 8, desc64(vl + kk * 128, kDescHi), idesc_pv, kk ? 1u : acc0);
       };
       for (int w_item = blockIdx.x; w_item < p.total_items && ok; w_item += gridDim.x, ++it) {
         const int item = w_item % p.items_per_kv, bh = w_item / p.items_per_kv;
         const Geo g = make_geo(p, item, bh % p.Hkv);
-        auto active = [&](int t, int j) {
-          return g.valid[t] && j < g.T && tile_class(p, g.q0[t], g.kstart + j * kTile) != kSkip;
-        };
-        int last[2] = {-1, -1};   // last active K/V tile of each query tile
+        // K/V tiles [first, last] that each query tile takes part in (a contiguous range)
+        int first[2] = {1 << 30, 1 << 30}, last[2] = {-1, -1};
         for (int t = 0; t < 2; ++t)
-          for (int j = g.T - 1; j >= 0; --j)
-            if (active(t, j)) { last[t] = j; break; }
-        int started[2] = {0, 0};
+          if (g.valid[t])
+            for (int j = 0; j < g.T; ++j)
+              if (tile_class(p, g.q0[t], g.kstart + j * kTile) != kSkip) {
+                first[t] = min(first[t], j);
+                last[t] = j;
+              }
+        auto active = [&](int t, int j) { return j >= first[t] && j <= last[t]; };
+        uint32_t started[2] = {0, 0};
         // ring uses of this item: K_j = use + 2j, V_j = use + 2j + 1
         ok = mbar_wait(bar(C::kBarQFull), it & 1u, gave_up, p.status);
         if (ok) ok = slot_wait(use);
         if (!ok) break;
+        fence_proxy_async();
         tc_fence_after();
         for (int t = 0; t < 2; ++t)
-          if (active(t, 0)) issue_qk(t, slot_addr(use));
+          if (active(t, 0)) issue_qk(t, slot_lo(use));
         tc_commit(bar(C::kBarSlotEmpty + use % C::kSlots));
         if (g.T == 1) tc_commit(bar(C::kBarQEmpty));
         for (int j = 0; j < g.T && ok; ++j) {
@@ -521,13 +516,9 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
               if (ok) ok = mbar_wait(bar(C::kBarPReady + t), p_cnt[t] & 1u, gave_up, p.status);
               if (!ok) break;
               ++p_cnt[t];
+              fence_proxy_async();
               tc_fence_after();
-              const uint32_t va = slot_addr(uv);
-#pragma unroll
-              for (int kk = 0; kk < kTile / 16; ++kk)
-                mma_ts(tmem + C::kColO + t * D, tmem + t * 128 + kk * 8,
-                       smem_desc(va + kk * 2048, C::kChunkBytes, 1024), idesc_pv,
-                       (started[t] | kk) != 0);
+              issue_pv(t, slot_lo(uv), started[t]);
               started[t] = 1;
               if (j == last[t]) tc_commit(bar(C::kBarODone + t));
             }
@@ -535,10 +526,11 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
               if (!k_ready) {
                 ok = slot_wait(uk);
                 if (!ok) break;
+                fence_proxy_async();
                 tc_fence_after();
                 k_ready = true;
               }
-              issue_qk(t, slot_addr(uk));
+              issue_qk(t, slot_lo(uk));
             }
           }
           if (ok && !v_ready) ok = slot_wait(uv);
