@@ -22,6 +22,8 @@
 //
 // Every mbarrier wait is bounded; on expiry the CTA records SA_ERR_TIMEOUT in the device
 // status word, stops issuing work, drains what it started and returns.
+#include <type_traits>
+
 #include "sa_fwd_tc.cuh"
 
 namespace sa {
@@ -29,6 +31,7 @@ namespace {
 
 constexpr int kTile = 128;           // query rows per tile and keys per K/V tile
 constexpr int kThreads = 384;
+constexpr int kHalf = 64;            // keys per score block (half a K/V tile)
 constexpr int kProducers = 96;       // threads of the three gather warps
 constexpr uint32_t kTmemCols = 512;
 constexpr long long kWaitCycles = 2000000000ll;  // about one second
@@ -152,13 +155,6 @@ __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32
       ::SA_W8(v, 0), SA_W8(v, 8), SA_W8(v, 16), SA_W8(v, 24), "r"(taddr)
       : "memory");
 }
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16]) {
-  asm volatile(
-      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%16], "
-      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15};"
-      ::SA_W8(v, 0), SA_W8(v, 8), "r"(taddr)
-      : "memory");
-}
 __device__ __forceinline__ void tmem_wait_ld() {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
@@ -199,8 +195,10 @@ struct Geo {
   int T;            // K/V tiles in the stream
 };
 
-__device__ __forceinline__ int tile_class(const TcParams& p, int q0, int kv) {
-  const int q1 = q0 + kTile - 1, k1 = kv + kTile - 1;
+// How the keys [kv, kv + kw) relate to the queries [q0, q0 + 128): not needed at all, all
+// visible, visible up to the token order only, or to be tested element by element.
+__device__ __forceinline__ int tile_class(const TcParams& p, int q0, int kv, int kw) {
+  const int q1 = q0 + kTile - 1, k1 = kv + kw - 1;
   if (p.full_range) return kv < p.n ? kEdge : kSkip;
   if (p.one_sided) {
     if (kv > q1 || k1 < q0 - (p.w - 1)) return kSkip;
@@ -285,8 +283,9 @@ struct Cfg {
   // mbarriers, 8 bytes each
   static constexpr int kBarQFull = 0, kBarQEmpty = 1, kBarSlotFull = 2,
                        kBarSlotEmpty = kBarSlotFull + kSlots, kBarTokFull = kBarSlotEmpty + kSlots,
-                       kBarSFull = kBarTokFull + kTok, kBarPReady = kBarSFull + 2,
-                       kBarODone = kBarPReady + 2, kNumBars = kBarODone + 2;
+                       kBarSFull = kBarTokFull + kTok, kBarPReady = kBarSFull + 4,
+                       kBarPvDone = kBarPReady + 4, kBarODone = kBarPvDone + 2,
+                       kNumBars = kBarODone + 2;
   static constexpr int kOffMisc = kOffBar + kNumBars * 8;   // TMEM base address, gave_up flag
   static constexpr int kBytes = kOffMisc + 16;
   static constexpr uint32_t kColO = 256;                     // O_t at 256 + t*D; S_t at t*128
@@ -318,7 +317,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
   if (threadIdx.x == 0) {
     *gave_up = 0;
     for (int i = 0; i < C::kNumBars; ++i)
-      mbar_init(bar(i), (i == C::kBarPReady || i == C::kBarPReady + 1) ? kTile
+      mbar_init(bar(i), (i >= C::kBarPReady && i < C::kBarPvDone) ? kTile
                         : (i == C::kBarQFull || (i >= C::kBarSlotFull && i < C::kBarSlotEmpty))
                             ? kProducers : 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -429,6 +428,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
           qtok[ptid + 96] = tq1;
           if (ptid < 64) qtok[ptid + 192] = tq2;
           if (group_sync_stop()) { live = false; break; }
+#pragma unroll
           for (int t = 0; t < 2; ++t)
             gather(qg + b * p.qs[0] + g.hq[t] * p.qs[1], p.qs[2], qtok + t * kTile,
                    sbase + C::kOffQ + t * C::kTileBytes);
@@ -449,8 +449,13 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
     // One thread feeds the tensor core, so every instruction between two tcgen05.mma counts:
     // the descriptors are built from words prepared outside the loops and the K steps are
     // fully unrolled with immediate offsets.
+    //
+    // Scores are produced 64 keys at a time into the two halves of a tile's S columns, two
+    // half-steps ahead of the softmax: while the softmax works on one half, the other half
+    // already holds the next scores, so the softmax never waits for Q K^T and the tensor
+    // core never waits for the softmax of the same tile.
     if (lane == 0) {
-      constexpr uint32_t idesc_qk = instr_desc(kTile, kTile, false);
+      constexpr uint32_t idesc_qk = instr_desc(kTile, kHalf, false);
       constexpr uint32_t idesc_pv = instr_desc(kTile, D, true);
       // shared-memory descriptor words (128-byte swizzle, 1024 bytes between 8-row groups)
       constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
@@ -461,84 +466,99 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
       const uint32_t ring_lo = (sbase + C::kOffRing) >> 4;
       bool ok = true;
       uint32_t use = 0, it = 0;
-      uint32_t p_cnt[2] = {0, 0};
+      uint32_t pc00 = 0, pc01 = 0, pc10 = 0, pc11 = 0;   // p_ready waits so far, per [tile][half]
       auto slot_lo = [&](uint32_t u) { return ring_lo + (u % C::kSlots) * (C::kTileBytes >> 4); };
       auto slot_wait = [&](uint32_t u) {
         return mbar_wait(bar(C::kBarSlotFull + u % C::kSlots), (u / C::kSlots) & 1u, gave_up,
                          p.status);
       };
-      auto issue_qk = [&](int t, uint32_t k_lo) {
-        const uint32_t ql = q_lo[t], kl = k_lo | kLoK, d = tmem + t * 128;
+      // S(t, half b) = Q_t K^T over keys [64 b, 64 b + 64) of the K tile at k_lo
+      auto issue_qk = [&](int t, int b, uint32_t k_lo) {
+        const uint32_t ql = q_lo[t], kl = (k_lo + b * (kHalf * 128 >> 4)) | kLoK;
+        const uint32_t d = tmem + t * 128 + b * kHalf;
 #pragma unroll
         for (int kk = 0; kk < D / 16; ++kk) {
           const uint32_t off = (kk / 4) * (C::kChunkBytes >> 4) + (kk % 4) * 2;
           mma_ss(d, desc64(ql + off, kDescHi), desc64(kl + off, kDescHi), idesc_qk, kk > 0);
         }
-        tc_commit(bar(C::kBarSFull + t));
+        tc_commit(bar(C::kBarSFull + 2 * t + b));
       };
-      auto issue_pv = [&](int t, uint32_t v_lo, uint32_t acc0) {
-        const uint32_t vl = v_lo | kLoV, d = tmem + C::kColO + t * D, a = tmem + t * 128;
+      // O_t += P(t, half b) V over the same 64 keys of the V tile at v_lo
+      auto issue_pv = [&](int t, int b, uint32_t v_lo, uint32_t acc0) {
+        const uint32_t vl = (v_lo + b * (kHalf * 128 >> 4)) | kLoV;
+        const uint32_t d = tmem + C::kColO + t * D, a = tmem + t * 128 + b * kHalf;
 #pragma unroll
-        for (int kk = 0; kk < kTile / 16; ++kk)
+        for (int kk = 0; kk < kHalf / 16; ++kk)
           mma_ts(d, a + kk * 8, desc64(vl + kk * 128, kDescHi), idesc_pv, kk ? 1u : acc0);
+        tc_commit(bar(C::kBarPvDone + t));
       };
       for (int w_item = blockIdx.x; w_item < p.total_items && ok; w_item += gridDim.x, ++it) {
         const int item = w_item % p.items_per_kv, bh = w_item / p.items_per_kv;
         const Geo g = make_geo(p, item, bh % p.Hkv);
-        // K/V tiles [first, last] that each query tile takes part in (a contiguous range)
-        int first[2] = {1 << 30, 1 << 30}, last[2] = {-1, -1};
-        for (int t = 0; t < 2; ++t)
-          if (g.valid[t])
-            for (int j = 0; j < g.T; ++j)
-              if (tile_class(p, g.q0[t], g.kstart + j * kTile) != kSkip) {
-                first[t] = min(first[t], j);
-                last[t] = j;
-              }
-        auto active = [&](int t, int j) { return j >= first[t] && j <= last[t]; };
-        uint32_t started[2] = {0, 0};
+        const int H = 2 * g.T;          // half-steps of this item
+        // half-steps [first, last] that each query tile takes part in (a contiguous range);
+        // everything per tile is kept in scalars so that nothing is indexed at run time
+        int first0 = 1 << 30, first1 = 1 << 30, last0 = -1, last1 = -1;
+        for (int h = 0; h < H; ++h) {
+          if (g.valid[0] && tile_class(p, g.q0[0], g.kstart + h * kHalf, kHalf) != kSkip) {
+            first0 = min(first0, h);
+            last0 = h;
+          }
+          if (g.valid[1] && tile_class(p, g.q0[1], g.kstart + h * kHalf, kHalf) != kSkip) {
+            first1 = min(first1, h);
+            last1 = h;
+          }
+        }
+        uint32_t started0 = 0, started1 = 0;
         // ring uses of this item: K_j = use + 2j, V_j = use + 2j + 1
         ok = mbar_wait(bar(C::kBarQFull), it & 1u, gave_up, p.status);
         if (ok) ok = slot_wait(use);
         if (!ok) break;
         fence_proxy_async();
         tc_fence_after();
-        for (int t = 0; t < 2; ++t)
-          if (active(t, 0)) issue_qk(t, slot_lo(use));
+        {
+          const uint32_t k0 = slot_lo(use);
+          if (first0 <= 0 && last0 >= 0) issue_qk(0, 0, k0);
+          if (first1 <= 0 && last1 >= 0) issue_qk(1, 0, k0);
+          if (first0 <= 1 && last0 >= 1) issue_qk(0, 1, k0);
+          if (first1 <= 1 && last1 >= 1) issue_qk(1, 1, k0);
+        }
         tc_commit(bar(C::kBarSlotEmpty + use % C::kSlots));
         if (g.T == 1) tc_commit(bar(C::kBarQEmpty));
         for (int j = 0; j < g.T && ok; ++j) {
           const uint32_t uv = use + 2 * j + 1, uk = use + 2 * j + 2;
-          const bool have_next = j + 1 < g.T;
-          bool k_ready = false, v_ready = false;
-          for (int t = 0; t < 2 && ok; ++t) {
-            if (active(t, j)) {
-              if (!v_ready) { ok = slot_wait(uv); v_ready = true; }
-              if (ok) ok = mbar_wait(bar(C::kBarPReady + t), p_cnt[t] & 1u, gave_up, p.status);
-              if (!ok) break;
-              ++p_cnt[t];
-              fence_proxy_async();
+          const bool more = j + 1 < g.T;
+          // first touch of V_j and of K_{j+1}: both are needed within this step
+          ok = slot_wait(uv);
+          if (ok && more) ok = slot_wait(uk);
+          if (!ok) break;
+          fence_proxy_async();
+          const uint32_t v_lo = slot_lo(uv), k_lo = slot_lo(uk);
+          // one (tile, half) unit: P V of half-step h, then Q K^T of half-step h + 2
+          auto unit = [&](auto tc, auto bc, int first, int last, uint32_t& started, uint32_t& pcnt) {
+            constexpr int t = decltype(tc)::value, b = decltype(bc)::value;
+            const int h = 2 * j + b;
+            if (h >= first && h <= last) {
+              ok = mbar_wait(bar(C::kBarPReady + 2 * t + b), pcnt & 1u, gave_up, p.status);
+              if (!ok) return;
+              ++pcnt;
               tc_fence_after();
-              issue_pv(t, slot_lo(uv), started[t]);
-              started[t] = 1;
-              if (j == last[t]) tc_commit(bar(C::kBarODone + t));
+              issue_pv(t, b, v_lo, started);
+              started = 1;
+              if (h == last) tc_commit(bar(C::kBarODone + t));
             }
-            if (have_next && active(t, j + 1)) {
-              if (!k_ready) {
-                ok = slot_wait(uk);
-                if (!ok) break;
-                fence_proxy_async();
-                tc_fence_after();
-                k_ready = true;
-              }
-              issue_qk(t, slot_lo(uk));
-            }
-          }
-          if (ok && !v_ready) ok = slot_wait(uv);
-          if (ok && have_next && !k_ready) ok = slot_wait(uk);
+            if (more && h + 2 >= first && h + 2 <= last) issue_qk(t, b, k_lo);
+          };
+          using I0 = std::integral_constant<int, 0>;
+          using I1 = std::integral_constant<int, 1>;
+          unit(I0{}, I0{}, first0, last0, started0, pc00);
+          if (ok) unit(I1{}, I0{}, first1, last1, started1, pc10);
+          if (ok) unit(I0{}, I1{}, first0, last0, started0, pc01);
+          if (ok) unit(I1{}, I1{}, first1, last1, started1, pc11);
           if (!ok) break;
           // the slots free when the products issued so far have finished
           tc_commit(bar(C::kBarSlotEmpty + uv % C::kSlots));
-          if (have_next) tc_commit(bar(C::kBarSlotEmpty + uk % C::kSlots));
+          if (more) tc_commit(bar(C::kBarSlotEmpty + uk % C::kSlots));
           if (j + 2 == g.T) tc_commit(bar(C::kBarQEmpty));
         }
         use += 2 * g.T;
@@ -554,46 +574,73 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
     const uint32_t lane_addr = (uint32_t)(row & ~31) << 16;
     const uint32_t s_addr = tmem + lane_addr + t * 128;
     const uint32_t o_addr = tmem + lane_addr + C::kColO + t * D;
-    uint32_t s_cnt = 0, o_cnt = 0, gt = 0;
+    uint32_t s_cnt0 = 0, s_cnt1 = 0, o_cnt = 0, pv_cnt = 0, gt = 0;
     bool ok = true;
 
-    for (int w_item = blockIdx.x; w_item < p.total_items && ok; w_item += gridDim.x) {
+    // geometry and query token of an item; fetched one item ahead
+    struct ItemCtx { int b, q0, hq, valid, kstart, T, q_tok; bool row_valid; };
+    auto load_item = [&](int w_item) {
+      ItemCtx c;
       const int item = w_item % p.items_per_kv, bh = w_item / p.items_per_kv;
-      const int hk = bh % p.Hkv, b = bh / p.Hkv;
-      const Geo g = make_geo(p, item, hk);
+      c.b = bh / p.Hkv;
+      const Geo g = make_geo(p, item, bh % p.Hkv);
+      c.q0 = t ? g.q0[1] : g.q0[0];
+      c.hq = t ? g.hq[1] : g.hq[0];
+      c.valid = t ? g.valid[1] : g.valid[0];
+      c.kstart = g.kstart;
+      c.T = g.T;
+      const int qv = c.q0 + row;
+      c.row_valid = c.valid && qv < p.n;
+      c.q_tok = c.row_valid ? (p.perm ? p.perm[(size_t)c.b * p.n + qv] : qv) : 0;
+      return c;
+    };
+    ItemCtx nxt{};
+    if ((int)blockIdx.x < p.total_items) nxt = load_item(blockIdx.x);
+
+    for (int w_item = blockIdx.x; w_item < p.total_items && ok; w_item += gridDim.x) {
+      const ItemCtx cur = nxt;
+      const int b = cur.b, q0 = cur.q0;
       const uint32_t gt0 = gt;
-      gt += g.T;
-      if (!g.valid[t]) continue;
-      const int32_t* perm = p.perm ? p.perm + (size_t)b * p.n : nullptr;
-      const int qv = g.q0[t] + row;
-      const bool row_valid = qv < p.n;
-      const int q_tok = row_valid ? (perm ? perm[qv] : qv) : 0;
+      gt += cur.T;
+      if (!cur.valid) {
+        if (w_item + (int)gridDim.x < p.total_items) nxt = load_item(w_item + gridDim.x);
+        continue;
+      }
+      const int qv = q0 + row;
+      const bool row_valid = cur.row_valid;
+      const int q_tok = cur.q_tok;
       const int qcmp = (p.causal && !p.one_sided) ? q_tok : 0x7fffffff;
       float m = -INFINITY, l = 0.f;
       bool started = false;
+      const int H = 2 * cur.T;
 
-      for (int j = 0; j < g.T; ++j) {
-        const int kv = g.kstart + j * kTile;
-        const int cls = tile_class(p, g.q0[t], kv);
+      for (int h = 0; h < H; ++h) {
+        const int kv = cur.kstart + h * kHalf;
+        const int cls = tile_class(p, q0, kv, kHalf);
         if (cls == kSkip) continue;
-        const uint32_t tg = gt0 + j;
+        const int hb = h & 1;
+        const uint32_t tg = gt0 + (h >> 1);
         ok = mbar_wait(bar(C::kBarTokFull + tg % C::kTok), (tg / C::kTok) & 1u, gave_up, p.status);
-        if (ok) ok = mbar_wait(bar(C::kBarSFull + t), s_cnt & 1u, gave_up, p.status);
+        if (ok)
+          ok = mbar_wait(bar(C::kBarSFull + 2 * t + hb), (hb ? s_cnt1 : s_cnt0) & 1u, gave_up,
+                         p.status);
         ok = __all_sync(0xffffffffu, ok);   // the tensor-memory loads below are warp-collective
         if (!ok) break;
-        ++s_cnt;
+        s_cnt0 += 1 - hb;
+        s_cnt1 += hb;
         tc_fence_after();
 
-        uint32_t sr[kTile];
+        const uint32_t sh_addr = s_addr + hb * kHalf;
+        uint32_t sr[kHalf];
 #pragma unroll
-        for (int c = 0; c < 4; ++c)
-          tmem_ld32(s_addr + 32 * c, reinterpret_cast<uint32_t(&)[32]>(sr[32 * c]));
+        for (int c = 0; c < kHalf / 32; ++c)
+          tmem_ld32(sh_addr + 32 * c, reinterpret_cast<uint32_t(&)[32]>(sr[32 * c]));
         tmem_wait_ld();
         const int32_t* ktok = reinterpret_cast<const int32_t*>(smem + C::kOffTok) +
-                              (tg % C::kTok) * kTile;
+                              (tg % C::kTok) * kTile + hb * kHalf;
         if (cls == kCausalOnly) {
 #pragma unroll
-          for (int c = 0; c < kTile; c += 4) {
+          for (int c = 0; c < kHalf; c += 4) {
             const int4 kt = *reinterpret_cast<const int4*>(ktok + c);
             if (kt.x > qcmp) sr[c] = 0xff800000u;
             if (kt.y > qcmp) sr[c + 1] = 0xff800000u;
@@ -613,7 +660,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
           if (hi < lo) { lo = 1 << 30; hi = lo; }
           const uint32_t span = (uint32_t)(hi - lo);
 #pragma unroll
-          for (int c = 0; c < kTile; c += 4) {
+          for (int c = 0; c < kHalf; c += 4) {
             const int4 kt = *reinterpret_cast<const int4*>(ktok + c);
             if ((uint32_t)(c - lo) > span || kt.x > qcmp) sr[c] = 0xff800000u;
             if ((uint32_t)(c + 1 - lo) > span || kt.y > qcmp) sr[c + 1] = 0xff800000u;
@@ -623,9 +670,9 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
         }
         float mx0 = __uint_as_float(sr[0]), mx1 = __uint_as_float(sr[1]);
 #pragma unroll
-        for (int c = 2; c < kTile; c += 4) {
+        for (int c = 2; c < kHalf; c += 4) {
           mx0 = max3(mx0, __uint_as_float(sr[c]), __uint_as_float(sr[c + 1]));
-          if (c + 2 < kTile)
+          if (c + 2 < kHalf)
             mx1 = max3(mx1, __uint_as_float(sr[c + 2]), __uint_as_float(sr[c + 3]));
         }
         const float m_new = fmaxf(m, fmaxf(mx0, mx1));
@@ -634,6 +681,11 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
         if (!started) {
           m = m_new;
         } else if (__any_sync(0xffffffffu, grow)) {
+          // O is still being accumulated by the previous P V: wait for it before touching O
+          ok = mbar_wait(bar(C::kBarPvDone + t), (pv_cnt - 1) & 1u, gave_up, p.status);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) break;
+          tc_fence_after();
           const float f = grow ? exp2f((m - m_new) * p.scale2) : 1.f;
           if (grow) { l *= f; m = m_new; }
 #pragma unroll
@@ -650,27 +702,26 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
         const float neg = (m == -INFINITY) ? 0.f : -m * p.scale2;
         const float2 sc2 = make_float2(p.scale2, p.scale2), ng2 = make_float2(neg, neg);
         float2 lsum = make_float2(0.f, 0.f);
+        uint32_t pk[kHalf / 2];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          uint32_t pk[16];
-#pragma unroll
-          for (int x = 0; x < 16; ++x) {
-            const float2 a = __ffma2_rn(make_float2(__uint_as_float(sr[32 * c + 2 * x]),
-                                                    __uint_as_float(sr[32 * c + 2 * x + 1])),
-                                        sc2, ng2);
-            const float2 e = make_float2(exp2f(a.x), exp2f(a.y));
-            lsum = __fadd2_rn(lsum, e);
-            const __nv_bfloat162 h2 = __floats2bfloat162_rn(e.x, e.y);
-            pk[x] = *reinterpret_cast<const uint32_t*>(&h2);
-          }
-          tmem_st16(s_addr + 16 * c, pk);
+        for (int x = 0; x < kHalf / 2; ++x) {
+          const float2 a = __ffma2_rn(make_float2(__uint_as_float(sr[2 * x]),
+                                                  __uint_as_float(sr[2 * x + 1])), sc2, ng2);
+          const float2 e = make_float2(exp2f(a.x), exp2f(a.y));
+          lsum = __fadd2_rn(lsum, e);
+          const __nv_bfloat162 h2 = __floats2bfloat162_rn(e.x, e.y);
+          pk[x] = *reinterpret_cast<const uint32_t*>(&h2);
         }
+        tmem_st32(sh_addr, pk);
         l += lsum.x + lsum.y;
         tmem_wait_st();
         tc_fence_before();
-        mbar_arrive(bar(C::kBarPReady + t));
+        mbar_arrive(bar(C::kBarPReady + 2 * t + hb));
+        ++pv_cnt;                           // the issuer answers every arrive with one P V
       }
       if (!ok) break;
+      // fetch the next item's geometry and query token while the last products finish
+      if (w_item + (int)gridDim.x < p.total_items) nxt = load_item(w_item + gridDim.x);
 
       ok = mbar_wait(bar(C::kBarODone + t), o_cnt & 1u, gave_up, p.status);
       ok = __all_sync(0xffffffffu, ok);
@@ -679,7 +730,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
       tc_fence_after();
       const float inv_l = 1.f / l;
       float g_this = 1.f, g_other = 0.f;
-      const int hq = g.hq[t];
+      const int hq = cur.hq;
       if (p.gate_logits) {
         const float s_sa = 1.f / (1.f + __expf(-p.gate_logits[hq]));
         const float s_swa = 1.f / (1.f + __expf(-p.gate_logits[p.Hq + hq]));
