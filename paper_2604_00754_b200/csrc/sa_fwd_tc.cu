@@ -113,22 +113,39 @@ __device__ __forceinline__ void tc_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
                ::"r"(bar) : "memory");
 }
-// D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void mma_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc,
-                                       uint32_t acc) {
+// Four consecutive K steps (16 elements each) of D (+)= A B^T with both operands in shared
+// memory; each step moves both descriptors on by 32 bytes inside the 128-byte swizzle row.
+// Written as one block so that the issuing thread spends three instructions per product.
+__device__ __forceinline__ void mma_ss_x4(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc,
+                                          uint32_t acc0) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(acc)
+      "{\n\t.reg .pred p0, p1;\n\t.reg .b64 a1, a2, a3, b1, b2, b3;\n\t"
+      "setp.ne.b32 p0, %4, 0;\n\tsetp.eq.b32 p1, %3, %3;\n\t"
+      "add.u64 a1, %1, 2;\n\tadd.u64 b1, %2, 2;\n\t"
+      "add.u64 a2, %1, 4;\n\tadd.u64 b2, %2, 4;\n\t"
+      "add.u64 a3, %1, 6;\n\tadd.u64 b3, %2, 6;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], a1, b1, %3, p1;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], a2, b2, %3, p1;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], a3, b3, %3, p1;\n\t}"
+      ::"r"(d), "l"(a), "l"(b), "r"(idesc), "r"(acc0)
       : "memory");
 }
-// D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void mma_ts(uint32_t d, uint32_t a, uint64_t b, uint32_t idesc,
-                                       uint32_t acc) {
+// Four consecutive K steps of D (+)= A B with A (bf16 pairs, 8 columns per step) in tensor
+// memory and B in shared memory, 16 rows (2048 bytes) further on each step.
+__device__ __forceinline__ void mma_ts_x4(uint32_t d, uint32_t a, uint64_t b, uint32_t idesc,
+                                          uint32_t acc0) {
   asm volatile(
-      "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-      ::"r"(d), "r"(a), "l"(b), "r"(idesc), "r"(acc)
+      "{\n\t.reg .pred p0, p1;\n\t.reg .b64 b1, b2, b3;\n\t.reg .b32 a1, a2, a3;\n\t"
+      "setp.ne.b32 p0, %4, 0;\n\tsetp.eq.b32 p1, %3, %3;\n\t"
+      "add.u32 a1, %1, 8;\n\tadd.u64 b1, %2, 128;\n\t"
+      "add.u32 a2, %1, 16;\n\tadd.u64 b2, %2, 256;\n\t"
+      "add.u32 a3, %1, 24;\n\tadd.u64 b3, %2, 384;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [a1], b1, %3, p1;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [a2], b2, %3, p1;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [a3], b3, %3, p1;\n\t}"
+      ::"r"(d), "r"(a), "l"(b), "r"(idesc), "r"(acc0)
       : "memory");
 }
 
@@ -213,6 +230,21 @@ __device__ __forceinline__ int tile_class(const TcParams& p, int q0, int kv, int
   // plain SWA: keys wholly before the queries need no causal test (no wrap inside)
   if (p.swa && kv >= 0 && k1 <= q0) return kFull;
   return kCausalOnly;
+}
+
+// The half-steps h (keys kstart + 64 h ... + 63) that tile_class does not skip for the
+// query tile at q0: a contiguous range [first, last], empty (first > last) for a tile
+// that does not exist.
+__device__ __forceinline__ void active_halves(const TcParams& p, int q0, int valid, int kstart,
+                                              int H, int* first, int* last) {
+  const int q1 = q0 + kTile - 1;
+  int lo, hi;   // keys of interest: some key of the half >= lo, its first key <= hi
+  if (p.full_range) { lo = 0; hi = p.n - 1; }
+  else if (p.one_sided) { lo = q0 - (p.w - 1); hi = q1; }
+  else { lo = q0 - p.h; hi = q1 + p.h; }
+  const int f = max(0, (lo - kstart) >> 6), l = min(H - 1, (hi - kstart) >> 6);
+  *first = valid ? f : (1 << 30);
+  *last = valid ? l : -1;
 }
 
 __device__ __forceinline__ Geo make_geo(const TcParams& p, int item, int hk) {
@@ -461,8 +493,8 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
       constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
       constexpr uint32_t kLoK = (16u >> 4) << 16;                          // K-major operands
       constexpr uint32_t kLoV = ((uint32_t)C::kChunkBytes >> 4) << 16;     // V: next 64 columns
-      const uint32_t q_lo[2] = {((sbase + C::kOffQ) >> 4) | kLoK,
-                                ((sbase + C::kOffQ + C::kTileBytes) >> 4) | kLoK};
+      const uint64_t q_desc0 = desc64(((sbase + C::kOffQ) >> 4) | kLoK, kDescHi);
+      const uint64_t q_desc1 = desc64(((sbase + C::kOffQ + C::kTileBytes) >> 4) | kLoK, kDescHi);
       const uint32_t ring_lo = (sbase + C::kOffRing) >> 4;
       bool ok = true;
       uint32_t use = 0, it = 0;
@@ -474,22 +506,18 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
       };
       // S(t, half b) = Q_t K^T over keys [64 b, 64 b + 64) of the K tile at k_lo
       auto issue_qk = [&](int t, int b, uint32_t k_lo) {
-        const uint32_t ql = q_lo[t], kl = (k_lo + b * (kHalf * 128 >> 4)) | kLoK;
+        const uint64_t qd = t ? q_desc1 : q_desc0;
+        const uint64_t kd = desc64((k_lo + b * (kHalf * 128 >> 4)) | kLoK, kDescHi);
         const uint32_t d = tmem + t * 128 + b * kHalf;
-#pragma unroll
-        for (int kk = 0; kk < D / 16; ++kk) {
-          const uint32_t off = (kk / 4) * (C::kChunkBytes >> 4) + (kk % 4) * 2;
-          mma_ss(d, desc64(ql + off, kDescHi), desc64(kl + off, kDescHi), idesc_qk, kk > 0);
-        }
+        mma_ss_x4(d, qd, kd, idesc_qk, 0u);
+        if (D == 128)   // columns 64..127 live one 16 KB block further on
+          mma_ss_x4(d, qd + (C::kChunkBytes >> 4), kd + (C::kChunkBytes >> 4), idesc_qk, 1u);
         tc_commit(bar(C::kBarSFull + 2 * t + b));
       };
       // O_t += P(t, half b) V over the same 64 keys of the V tile at v_lo
       auto issue_pv = [&](int t, int b, uint32_t v_lo, uint32_t acc0) {
-        const uint32_t vl = (v_lo + b * (kHalf * 128 >> 4)) | kLoV;
-        const uint32_t d = tmem + C::kColO + t * D, a = tmem + t * 128 + b * kHalf;
-#pragma unroll
-        for (int kk = 0; kk < kHalf / 16; ++kk)
-          mma_ts(d, a + kk * 8, desc64(vl + kk * 128, kDescHi), idesc_pv, kk ? 1u : acc0);
+        const uint64_t vd = desc64((v_lo + b * (kHalf * 128 >> 4)) | kLoV, kDescHi);
+        mma_ts_x4(tmem + C::kColO + t * D, tmem + t * 128 + b * kHalf, vd, idesc_pv, acc0);
         tc_commit(bar(C::kBarPvDone + t));
       };
       for (int w_item = blockIdx.x; w_item < p.total_items && ok; w_item += gridDim.x, ++it) {
@@ -498,17 +526,9 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
         const int H = 2 * g.T;          // half-steps of this item
         // half-steps [first, last] that each query tile takes part in (a contiguous range);
         // everything per tile is kept in scalars so that nothing is indexed at run time
-        int first0 = 1 << 30, first1 = 1 << 30, last0 = -1, last1 = -1;
-        for (int h = 0; h < H; ++h) {
-          if (g.valid[0] && tile_class(p, g.q0[0], g.kstart + h * kHalf, kHalf) != kSkip) {
-            first0 = min(first0, h);
-            last0 = h;
-          }
-          if (g.valid[1] && tile_class(p, g.q0[1], g.kstart + h * kHalf, kHalf) != kSkip) {
-            first1 = min(first1, h);
-            last1 = h;
-          }
-        }
+        int first0, first1, last0, last1;
+        active_halves(p, g.q0[0], g.valid[0], g.kstart, H, &first0, &last0);
+        active_halves(p, g.q0[1], g.valid[1], g.kstart, H, &first1, &last1);
         uint32_t started0 = 0, started1 = 0;
         // ring uses of this item: K_j = use + 2j, V_j = use + 2j + 1
         ok = mbar_wait(bar(C::kBarQFull), it & 1u, gave_up, p.status);
@@ -578,7 +598,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
     bool ok = true;
 
     // geometry and query token of an item; fetched one item ahead
-    struct ItemCtx { int b, q0, hq, valid, kstart, T, q_tok; bool row_valid; };
+    struct ItemCtx { int b, q0, hq, valid, kstart, T, first, last, q_tok; bool row_valid; };
     auto load_item = [&](int w_item) {
       ItemCtx c;
       const int item = w_item % p.items_per_kv, bh = w_item / p.items_per_kv;
@@ -589,6 +609,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
       c.valid = t ? g.valid[1] : g.valid[0];
       c.kstart = g.kstart;
       c.T = g.T;
+      active_halves(p, c.q0, c.valid, c.kstart, 2 * c.T, &c.first, &c.last);
       const int qv = c.q0 + row;
       c.row_valid = c.valid && qv < p.n;
       c.q_tok = c.row_valid ? (p.perm ? p.perm[(size_t)c.b * p.n + qv] : qv) : 0;
@@ -612,12 +633,10 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
       const int qcmp = (p.causal && !p.one_sided) ? q_tok : 0x7fffffff;
       float m = -INFINITY, l = 0.f;
       bool started = false;
-      const int H = 2 * cur.T;
 
-      for (int h = 0; h < H; ++h) {
+      for (int h = cur.first; h <= cur.last; ++h) {
         const int kv = cur.kstart + h * kHalf;
         const int cls = tile_class(p, q0, kv, kHalf);
-        if (cls == kSkip) continue;
         const int hb = h & 1;
         const uint32_t tg = gt0 + (h >> 1);
         ok = mbar_wait(bar(C::kBarTokFull + tg % C::kTok), (tg / C::kTok) & 1u, gave_up, p.status);
