@@ -7,6 +7,9 @@
 //               over the query heads of its GQA group.
 // Formulas: derivative of Eq. 1 / Eq. 5 with the permutation held constant,
 //   P_ij = exp(scale q_i.k_j - lse_i), dS_ij = P_ij (dY_x[i].V_j - D_x[i]).
+#include <type_traits>
+
+#include "sa_bwd_tc.cuh"
 #include "sa_common.cuh"
 
 namespace sa {
@@ -241,6 +244,8 @@ cudaError_t launch_all(const BwdArgs& a, cudaStream_t st) {
     dgate_kernel<<<(2 * a.Hq + 127) / 128, 128, 0, st>>>(a);
     bump_launches();
   }
+  if (tc_backward_supported(a, std::is_same<T, float>::value ? SA_F32 : SA_BF16))
+    return launch_bwd_tc(a, st);      // dq, dk, dv on the tensor cores
   bwd_dq_kernel<T><<<dim3((a.n + kWarps - 1) / kWarps, a.Hq, a.B), kWarps * 32, smem, st>>>(a);
   bwd_dkv_kernel<T><<<dim3((a.n + kWarps - 1) / kWarps, a.Hkv, a.B), kWarps * 32, smem, st>>>(a);
   bump_launches(2);

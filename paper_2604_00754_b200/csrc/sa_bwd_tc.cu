@@ -1,0 +1,491 @@
+// Backward pass on the 5th-generation tensor cores, bf16, d = 64 or 128.
+//
+// Formulas (derivative of Eq. 1 with the permutation held constant; per branch x, with
+// dO = g_x dY and Delta_i = g_x sum_c dY[i,c] Y_x[i,c] prepared by the delta kernel):
+//   P_ij = exp(scale q_i.k_j - lse_i),  dP_ij = dY_i . v_j,
+//   dS_ij = scale P_ij (g_x dP_ij - Delta_i),
+//   dQ_i = sum_j dS_ij k_j,   dK_j = sum_i dS_ij q_i,   dV_j = sum_i g_x P_ij dY_i.
+//
+// Two launches per branch, neither of which needs an atomic, so results are run-to-run
+// identical:
+//   rows = queries: a CTA owns 128 query slots of one head, walks the K/V tiles of its
+//                   band, and accumulates dQ;
+//   rows = keys:    a CTA owns 128 key slots of one KV head, walks the query tiles that can
+//                   see them for every query head of the group, and accumulates dK and dV.
+// Either way one step is: S = R1 C1^T and dP = R2 C2^T into tensor memory (rows: Q, dY or
+// K, V; columns: K, V or Q, dY), one thread per row turns them into P and dS (bf16, written
+// back over S and dP), then dS (and P) multiply the column tiles into the accumulators.
+// Rows of every operand are gathered through perm with cp.async into swizzled shared
+// memory, as in the forward kernel; finished rows are scattered to their original places.
+//
+// Warp roles (256 threads): warp 0 MMA issuer and TMEM allocator, warps 1-3 gather
+// producers, warps 4-7 one thread per row.  Every mbarrier wait is bounded.
+#include "sa_bwd_tc.cuh"
+#include "sa_tc_common.cuh"
+
+namespace sa {
+namespace {
+
+constexpr int kTile = 128;
+constexpr int kBwdThreads = 256;
+constexpr int kProducers = 96;
+constexpr uint32_t kTmemCols = 512;
+
+struct BwdTcParams {
+  const void *q, *k, *v, *dy;
+  const int32_t* perm;        // null for the SWA branch
+  const float* lse;           // [B,Hq,n] of this branch
+  const float* delta;         // [B,Hq,n] of this branch (gate included)
+  const float* gate_logit;    // null, or the [Hq] logits of this branch
+  void *dq, *dk, *dv;
+  int accumulate;             // add to what the outputs already hold
+  int* status;
+  const int* abort_flag;
+  int B, Hq, Hkv, G, n, w, h;
+  int causal, linear, one_sided, full_range;
+  int n_tiles;
+  float scale, scale2;
+  int64_t qs[3], ks[3];
+};
+
+// Columns (virtual slots) a row tile starting at slot r0 has to meet: [cstart, cend].
+// rows_are_keys selects the transposed window of the one-sided rule.
+__device__ __forceinline__ void column_range(const BwdTcParams& p, int r0, bool rows_are_keys,
+                                             int* cstart, int* T) {
+  const int rl = min(r0 + kTile - 1, p.n - 1);
+  int lo, hi;
+  if (p.full_range) { lo = 0; hi = p.n - 1; }
+  else if (p.one_sided) {
+    if (rows_are_keys) { lo = r0; hi = min(rl + p.w - 1, p.n - 1); }
+    else { lo = max(r0 - (p.w - 1), 0); hi = rl; }
+  } else if (p.linear) { lo = max(r0 - p.h, 0); hi = min(rl + p.h, p.n - 1); }
+  else { lo = r0 - p.h; hi = rl + p.h; }
+  *cstart = lo;
+  *T = (hi - lo + kTile) / kTile;
+}
+
+__device__ __forceinline__ int actual_slot(const BwdTcParams& p, int v) {
+  if (p.full_range || p.linear || p.one_sided) return min(max(v, 0), p.n - 1);
+  v %= p.n;
+  return v < 0 ? v + p.n : v;
+}
+
+template <int D>
+struct BCfg {
+  static constexpr int kTileBytes = kTile * D * 2;
+  static constexpr int kChunkBytes = kTile * 128;
+  static constexpr int kStages = 2;
+  static constexpr int kOffR = 0;                               // two row-operand tiles
+  static constexpr int kOffC = 2 * kTileBytes;                  // kStages x two column tiles
+  static constexpr int kOffRowTok = kOffC + kStages * 2 * kTileBytes;
+  static constexpr int kOffColTok = kOffRowTok + kTile * 4;     // kStages x 128 ints
+  static constexpr int kOffColVec = kOffColTok + kStages * kTile * 4;  // kStages x 2 x 128 floats
+  static constexpr int kOffBar = kOffColVec + kStages * 2 * kTile * 4;
+  static constexpr int kBarRFull = 0, kBarCFull = 1, kBarCEmpty = kBarCFull + kStages,
+                       kBarTokFull = kBarCEmpty + kStages, kBarSFull = kBarTokFull + kStages,
+                       kBarPReady = kBarSFull + 1, kBarODone = kBarPReady + 1,
+                       kNumBars = kBarODone + 1;
+  static constexpr int kOffMisc = kOffBar + kNumBars * 8;
+  static constexpr int kBytes = kOffMisc + 16;
+  // tensor memory columns: S and dS at 0, dP and P at 128, accumulators from 256
+  static constexpr uint32_t kColS = 0, kColP = 128, kColAcc = 256;
+  static_assert(kBytes <= 232448, "shared memory");
+};
+
+// MODE 0: rows are queries (dQ).  MODE 1: rows are keys (dK, dV).
+template <int D, int MODE>
+__global__ void __launch_bounds__(kBwdThreads, 1) bwd_tc_kernel(const __grid_constant__ BwdTcParams p) {
+  extern __shared__ __align__(1024) uint8_t smem[];
+  using C = BCfg<D>;
+  constexpr bool kKeys = MODE == 1;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (p.abort_flag && *p.abort_flag) return;  // an earlier check rejected perm/inv (uniform)
+  if (*(volatile int*)p.status == SA_ERR_TIMEOUT) return;
+  const uint32_t sbase = smem_u32(smem);
+  if (sbase & 1023u) {
+    if (threadIdx.x == 0) atomicCAS(p.status, SA_OK, SA_ERR_CUDA);
+    return;
+  }
+  const uint32_t bar0 = sbase + C::kOffBar;
+  auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + C::kOffMisc);
+  volatile int* gave_up = reinterpret_cast<volatile int*>(smem + C::kOffMisc + 4);
+
+  // work item: (batch, head of the row operand, row tile)
+  const int H = kKeys ? p.Hkv : p.Hq;
+  const int tile = blockIdx.x % p.n_tiles, bh = blockIdx.x / p.n_tiles;
+  const int hr = bh % H, b = bh / H;
+  const int hk = kKeys ? hr : hr / p.G;
+  const int r0 = tile * kTile;
+  int cstart, T;
+  column_range(p, r0, kKeys, &cstart, &T);
+  const int iters = kKeys ? T * p.G : T;      // column tiles (times query heads of the group)
+  const int32_t* perm = p.perm ? p.perm + (size_t)b * p.n : nullptr;
+
+  if (threadIdx.x == 0) {
+    *gave_up = 0;
+    for (int i = 0; i < C::kNumBars; ++i)
+      mbar_init(bar(i), i == C::kBarPReady ? kTile
+                        : (i == C::kBarRFull || (i >= C::kBarCFull && i < C::kBarCEmpty))
+                            ? kProducers : 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 0) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp >= 1 && warp < 4) {
+    // ---------------------------------------------------- gather producers (warps 1-3)
+    constexpr int kCpr = D / 8;            // 16-byte pieces per row
+    constexpr int kRpi = 32 / kCpr;        // rows per warp instruction
+    const int ptid = threadIdx.x - 32;     // 0..95
+    const int sub = lane / kCpr, chunk = lane % kCpr;
+    const uint32_t dst_lane = (uint32_t)(chunk >> 3) * C::kChunkBytes;
+    const __nv_bfloat16* qg = (const __nv_bfloat16*)p.q;
+    const __nv_bfloat16* kg = (const __nv_bfloat16*)p.k;
+    const __nv_bfloat16* vg = (const __nv_bfloat16*)p.v;
+    const __nv_bfloat16* dyg = (const __nv_bfloat16*)p.dy;
+    int32_t* const rowtok = reinterpret_cast<int32_t*>(smem + C::kOffRowTok);
+    auto signal = [&](uint32_t mb) {
+      asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(mb) : "memory");
+    };
+    auto gather = [&](const __nv_bfloat16* base, int64_t tok_stride, const int32_t* toks,
+                      uint32_t dst_tile) {
+#pragma unroll 4
+      for (int grp = warp - 1; grp < kTile / kRpi; grp += 3) {
+        const int r = grp * kRpi + sub;
+        const __nv_bfloat16* src = base + (int64_t)toks[r] * tok_stride + chunk * 8;
+        const uint32_t dst = dst_tile + dst_lane + r * 128 + (((chunk & 7) ^ (r & 7)) << 4);
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+      }
+    };
+    // Barrier over the three producer warps that also agrees on whether anyone in the CTA
+    // has given up, so that every producer thread leaves at the same point.
+    auto group_sync_stop = [&]() {
+      uint32_t any;
+      asm volatile(
+          "{\n\t.reg .pred p, q;\n\t"
+          "setp.ne.u32 q, %1, 0;\n\t"
+          "bar.red.or.pred p, 1, 96, q;\n\t"
+          "selp.u32 %0, 1, 0, p;\n\t}"
+          : "=r"(any)
+          : "r"((uint32_t)*gave_up)
+          : "memory");
+      return any != 0;
+    };
+    auto tok_of = [&](int slot) { return perm ? perm[slot] : slot; };
+
+    // row operands
+    rowtok[ptid] = tok_of(min(r0 + ptid, p.n - 1));
+    if (ptid < 32) rowtok[ptid + 96] = tok_of(min(r0 + ptid + 96, p.n - 1));
+    bool live = !group_sync_stop();
+    if (live) {
+      if (kKeys) {
+        gather(kg + b * p.ks[0] + hr * p.ks[1], p.ks[2], rowtok, sbase + C::kOffR);
+        gather(vg + b * p.ks[0] + hr * p.ks[1], p.ks[2], rowtok, sbase + C::kOffR + C::kTileBytes);
+      } else {
+        gather(qg + b * p.qs[0] + hr * p.qs[1], p.qs[2], rowtok, sbase + C::kOffR);
+        gather(dyg + b * p.qs[0] + hr * p.qs[1], p.qs[2], rowtok, sbase + C::kOffR + C::kTileBytes);
+      }
+      signal(bar(C::kBarRFull));
+    }
+    for (int it = 0; it < iters && live; ++it) {
+      const int s = it & 1;
+      const int j = kKeys ? it % T : it, gi = kKeys ? it / T : 0;
+      const int hq = kKeys ? hk * p.G + gi : hr;
+      if (it >= C::kStages)
+        mbar_wait(bar(C::kBarCEmpty + s), ((it >> 1) - 1) & 1u, gave_up, p.status);
+      int32_t* coltok = reinterpret_cast<int32_t*>(smem + C::kOffColTok) + s * kTile;
+      const uint32_t colvec = sbase + C::kOffColVec + s * 2 * kTile * 4;
+      const int t0 = tok_of(actual_slot(p, cstart + j * kTile + ptid));
+      coltok[ptid] = t0;
+      int t1 = 0;
+      if (ptid < 32) {
+        t1 = tok_of(actual_slot(p, cstart + j * kTile + ptid + 96));
+        coltok[ptid + 96] = t1;
+      }
+      if (group_sync_stop()) { live = false; break; }
+      if (ptid == 0) mbar_arrive(bar(C::kBarTokFull + s));
+      const uint32_t c1 = sbase + C::kOffC + s * 2 * C::kTileBytes, c2 = c1 + C::kTileBytes;
+      if (kKeys) {
+        // per-query vectors of this head travel with the tile
+        const float* lse_h = p.lse + ((size_t)b * p.Hq + hq) * p.n;
+        const float* del_h = p.delta + ((size_t)b * p.Hq + hq) * p.n;
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(colvec + 4 * ptid), "l"(lse_h + t0) : "memory");
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(colvec + 4 * (kTile + ptid)), "l"(del_h + t0) : "memory");
+        if (ptid < 32) {
+          asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(colvec + 4 * (ptid + 96)), "l"(lse_h + t1) : "memory");
+          asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(colvec + 4 * (kTile + ptid + 96)), "l"(del_h + t1) : "memory");
+        }
+        gather(qg + b * p.qs[0] + hq * p.qs[1], p.qs[2], coltok, c1);
+        gather(dyg + b * p.qs[0] + hq * p.qs[1], p.qs[2], coltok, c2);
+      } else {
+        gather(kg + b * p.ks[0] + hk * p.ks[1], p.ks[2], coltok, c1);
+        gather(vg + b * p.ks[0] + hk * p.ks[1], p.ks[2], coltok, c2);
+      }
+      signal(bar(C::kBarCFull + s));
+    }
+    asm volatile("cp.async.wait_all;" ::: "memory");   // nothing in flight when the CTA leaves
+  } else if (warp == 0) {
+    // -------------------------------------------------------------- MMA issuer (warp 0)
+    if (lane == 0) {
+      constexpr uint32_t idesc_s = instr_desc(kTile, kTile, false);
+      constexpr uint32_t idesc_acc = instr_desc(kTile, D, true);
+      constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
+      constexpr uint32_t kLoK = (16u >> 4) << 16;                        // K-major operands
+      constexpr uint32_t kLoMN = ((uint32_t)C::kChunkBytes >> 4) << 16;  // column tile as [k][n]
+      constexpr uint32_t kBlock = C::kChunkBytes >> 4;   // next 64 columns of a K-major tile
+      const uint64_t r1 = desc64(((sbase + C::kOffR) >> 4) | kLoK, kDescHi);
+      const uint64_t r2 = desc64(((sbase + C::kOffR + C::kTileBytes) >> 4) | kLoK, kDescHi);
+      // X (128 x 128, fp32, tensor memory column col) = A B^T, both tiles K-major, K = D
+      auto product = [&](uint32_t col, uint64_t a, uint32_t b_addr) {
+        const uint64_t bd = desc64((b_addr >> 4) | kLoK, kDescHi);
+        mma_ss_x4(tmem + col, a, bd, idesc_s, 0u);
+        if (D == 128) mma_ss_x4(tmem + col, a + kBlock, bd + kBlock, idesc_s, 1u);
+      };
+      // acc (128 x D, tensor memory column col) += X (bf16 pairs at column xcol) * tile
+      auto accumulate = [&](uint32_t col, uint32_t xcol, uint32_t b_addr, uint32_t acc0) {
+        const uint64_t bd = desc64((b_addr >> 4) | kLoMN, kDescHi);
+        mma_ts_x4(tmem + col, tmem + xcol, bd, idesc_acc, acc0);
+        mma_ts_x4(tmem + col, tmem + xcol + 32, bd + 512, idesc_acc, 1u);
+      };
+      bool ok = mbar_wait(bar(C::kBarRFull), 0, gave_up, p.status);
+      for (int it = 0; it < iters && ok; ++it) {
+        const int s = it & 1;
+        const uint32_t c1 = sbase + C::kOffC + s * 2 * C::kTileBytes, c2 = c1 + C::kTileBytes;
+        ok = mbar_wait(bar(C::kBarCFull + s), (it >> 1) & 1u, gave_up, p.status);
+        if (!ok) break;
+        fence_proxy_async();
+        tc_fence_after();
+        product(C::kColS, r1, c1);
+        product(C::kColP, r2, c2);
+        tc_commit(bar(C::kBarSFull));
+        ok = mbar_wait(bar(C::kBarPReady), it & 1u, gave_up, p.status);
+        if (!ok) break;
+        tc_fence_after();
+        if (kKeys) {
+          accumulate(C::kColAcc, C::kColP, c2, it > 0);        // dV += (g P)^T dY
+          accumulate(C::kColAcc + D, C::kColS, c1, it > 0);    // dK += dS^T Q
+        } else {
+          accumulate(C::kColAcc, C::kColS, c1, it > 0);        // dQ += dS K
+        }
+        tc_commit(bar(C::kBarCEmpty + s));
+      }
+      if (ok) tc_commit(bar(C::kBarODone));
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------- one thread per row (warps 4-7)
+    const int row = threadIdx.x - 128;                  // 0..127 == TMEM lane
+    const uint32_t trow = tmem + ((uint32_t)(row & ~31) << 16);
+    const int rslot = r0 + row;
+    const bool row_valid = rslot < p.n;
+    const int rtok = perm ? perm[min(rslot, p.n - 1)] : min(rslot, p.n - 1);
+    const bool tok_rule = p.causal && !p.one_sided;     // token order decides, not slots
+    // rows = queries: mask key tokens above the query's; rows = keys: query tokens below
+    const int cmp = tok_rule ? rtok : (kKeys ? (int)0x80000000 : 0x7fffffff);
+    float lse2_r = 0.f, delta_r = 0.f, g = 1.f;
+    if (!kKeys) {
+      const size_t o = ((size_t)b * p.Hq + hr) * p.n + rtok;
+      lse2_r = p.lse[o] * kLog2e;
+      delta_r = p.delta[o];
+      if (p.gate_logit) g = 1.f / (1.f + __expf(-p.gate_logit[hr]));
+    }
+    bool ok = true;
+    for (int it = 0; it < iters; ++it) {
+      const int s = it & 1;
+      const int j = kKeys ? it % T : it;
+      if (kKeys && p.gate_logit) g = 1.f / (1.f + __expf(-p.gate_logit[hk * p.G + it / T]));
+      ok = mbar_wait(bar(C::kBarTokFull + s), (it >> 1) & 1u, gave_up, p.status);
+      if (ok) ok = mbar_wait(bar(C::kBarSFull), it & 1u, gave_up, p.status);
+      ok = __all_sync(0xffffffffu, ok);   // the tensor-memory accesses below are warp-collective
+      if (!ok) break;
+      tc_fence_after();
+      // visible columns of this row: one interval [lo, lo + span], cut by the token order
+      const int cb = cstart + j * kTile;
+      int lo, hi;
+      if (p.one_sided) {
+        if (kKeys) { lo = rslot - cb; hi = p.full_range ? p.n - 1 - cb : rslot + (p.w - 1) - cb; }
+        else { lo = p.full_range ? -cb : rslot - (p.w - 1) - cb; hi = rslot - cb; }
+      } else if (p.full_range && !p.linear) { lo = -cb; hi = p.n - 1 - cb; }
+      else { lo = rslot - p.h - cb; hi = rslot + p.h - cb; }
+      if (p.linear || p.full_range || p.one_sided) {
+        lo = max(lo, -cb);
+        hi = min(hi, p.n - 1 - cb);
+      }
+      if (hi < lo) { lo = 1 << 30; hi = lo; }
+      const uint32_t span = (uint32_t)(hi - lo);
+      const int32_t* coltok = reinterpret_cast<const int32_t*>(smem + C::kOffColTok) + s * kTile;
+      const float* colvec = reinterpret_cast<const float*>(smem + C::kOffColVec) + s * 2 * kTile;
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
+        uint32_t sv[32], dv[32];
+        tmem_ld32(trow + C::kColS + 32 * c, sv);
+        tmem_ld32(trow + C::kColP + 32 * c, dv);
+        tmem_wait_ld();
+        uint32_t ds_pk[16], p_pk[16];
+#pragma unroll
+        for (int x = 0; x < 32; x += 4) {
+          const int col = 32 * c + x;
+          const int4 ct = *reinterpret_cast<const int4*>(coltok + col);
+          float4 l4 = make_float4(lse2_r, lse2_r, lse2_r, lse2_r);
+          float4 d4 = make_float4(delta_r, delta_r, delta_r, delta_r);
+          if (kKeys) {
+            l4 = *reinterpret_cast<const float4*>(colvec + col);
+            l4.x *= kLog2e; l4.y *= kLog2e; l4.z *= kLog2e; l4.w *= kLog2e;
+            d4 = *reinterpret_cast<const float4*>(colvec + kTile + col);
+          }
+          const int ctk[4] = {ct.x, ct.y, ct.z, ct.w};
+          const float lv[4] = {l4.x, l4.y, l4.z, l4.w}, dl[4] = {d4.x, d4.y, d4.z, d4.w};
+          float pv[4], dsv[4];
+#pragma unroll
+          for (int y = 0; y < 4; ++y) {
+            const bool vis = (uint32_t)(col + y - lo) <= span &&
+                             (kKeys ? ctk[y] >= cmp : ctk[y] <= cmp);
+            const float e = exp2f(fmaf(__uint_as_float(sv[x + y]), p.scale2, -lv[y]));
+            pv[y] = vis ? e : 0.f;
+            dsv[y] = pv[y] * (g * __uint_as_float(dv[x + y]) - dl[y]) * p.scale;
+            pv[y] *= g;
+          }
+          const __nv_bfloat162 a0 = __floats2bfloat162_rn(dsv[0], dsv[1]);
+          const __nv_bfloat162 a1 = __floats2bfloat162_rn(dsv[2], dsv[3]);
+          ds_pk[x / 2] = *reinterpret_cast<const uint32_t*>(&a0);
+          ds_pk[x / 2 + 1] = *reinterpret_cast<const uint32_t*>(&a1);
+          if (kKeys) {
+            const __nv_bfloat162 b0 = __floats2bfloat162_rn(pv[0], pv[1]);
+            const __nv_bfloat162 b1 = __floats2bfloat162_rn(pv[2], pv[3]);
+            p_pk[x / 2] = *reinterpret_cast<const uint32_t*>(&b0);
+            p_pk[x / 2 + 1] = *reinterpret_cast<const uint32_t*>(&b1);
+          }
+        }
+        // bf16 results go back over the columns already consumed (16 c .. 16 c + 15)
+        tmem_st16(trow + C::kColS + 16 * c, ds_pk);
+        if (kKeys) tmem_st16(trow + C::kColP + 16 * c, p_pk);
+      }
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(bar(C::kBarPReady));
+    }
+
+    if (ok) ok = mbar_wait(bar(C::kBarODone), 0, gave_up, p.status);
+    ok = __all_sync(0xffffffffu, ok);
+    if (ok) {
+      tc_fence_after();
+      constexpr int kOuts = kKeys ? 2 : 1;
+#pragma unroll
+      for (int o = 0; o < kOuts; ++o) {
+        // rows = keys: accumulator 0 is dV, 1 is dK
+        __nv_bfloat16* out = (__nv_bfloat16*)(kKeys ? (o == 0 ? p.dv : p.dk) : p.dq);
+        const int64_t* st = kKeys ? p.ks : p.qs;
+        const int64_t off = b * st[0] + hr * st[1] + (int64_t)rtok * st[2];
+#pragma unroll
+        for (int c = 0; c < D / 32; ++c) {
+          uint32_t raw[32];
+          tmem_ld32(trow + C::kColAcc + o * D + 32 * c, raw);   // warp-collective
+          tmem_wait_ld();
+          if (row_valid) {
+#pragma unroll
+            for (int x8 = 0; x8 < 4; ++x8) {
+              float v8[8];
+#pragma unroll
+              for (int x = 0; x < 8; ++x) v8[x] = __uint_as_float(raw[8 * x8 + x]);
+              uint4* dst = reinterpret_cast<uint4*>(out + off + 32 * c + 8 * x8);
+              if (p.accumulate) {
+                const uint4 old = *dst;
+                const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&old);
+#pragma unroll
+                for (int x = 0; x < 4; ++x) {
+                  v8[2 * x] += __low2float(h2[x]);
+                  v8[2 * x + 1] += __high2float(h2[x]);
+                }
+              }
+              uint4 pk;
+              __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&pk);
+#pragma unroll
+              for (int x = 0; x < 4; ++x) h2[x] = __floats2bfloat162_rn(v8[2 * x], v8[2 * x + 1]);
+              *dst = pk;
+            }
+          }
+        }
+      }
+    }
+  }
+
+  // ----------------------------------------------------------------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols)
+                 : "memory");
+  }
+}
+
+// ---------------------------------------------------------------------------- host
+
+template <int D>
+cudaError_t launch_branch(const BwdTcParams& p, cudaStream_t st) {
+  const int smem = BCfg<D>::kBytes;
+  cudaError_t e = cudaFuncSetAttribute(bwd_tc_kernel<D, 0>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(bwd_tc_kernel<D, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  if (e != cudaSuccess) return e;
+  bwd_tc_kernel<D, 0><<<(unsigned)(p.B * p.Hq * p.n_tiles), kBwdThreads, smem, st>>>(p);
+  bwd_tc_kernel<D, 1><<<(unsigned)(p.B * p.Hkv * p.n_tiles), kBwdThreads, smem, st>>>(p);
+  bump_launches(2);
+  return cudaGetLastError();
+}
+
+bool bwd_tc_disabled() {
+  static int v = -1;
+  if (v < 0) {
+    const char* e = getenv("SA_DISABLE_TC");
+    v = (e && e[0] == '1') ? 1 : 0;
+  }
+  return v == 1;
+}
+
+}  // namespace
+
+bool tc_backward_supported(const BwdArgs& a, int dtype) {
+  if (bwd_tc_disabled() || dtype != SA_BF16 || (a.d != 128 && a.d != 64)) return false;
+  return a.n >= 1 && (int64_t)a.B * a.Hq * ((a.n + kTile - 1) / kTile) <= 0x3fffffff;
+}
+
+cudaError_t launch_bwd_tc(const BwdArgs& a, cudaStream_t st) {
+  for (int x = 0; x < a.nbranch; ++x) {
+    BwdTcParams p{};
+    p.q = a.q; p.k = a.k; p.v = a.v; p.dy = a.dy;
+    p.perm = x == 0 ? a.perm : nullptr;
+    p.lse = a.lse_x[x];
+    p.delta = a.delta + (size_t)x * a.B * a.Hq * a.n;
+    p.gate_logit = a.gate_logits ? a.gate_logits + (size_t)x * a.Hq : nullptr;
+    p.dq = a.dq; p.dk = a.dk; p.dv = a.dv;
+    p.accumulate = x > 0;
+    p.status = status_ptr();
+    if (!p.status) return cudaErrorUnknown;
+    p.abort_flag = a.abort_flag;
+    p.B = a.B; p.Hq = a.Hq; p.Hkv = a.Hkv; p.G = a.Hq / a.Hkv; p.n = a.n; p.w = a.w;
+    const MaskGeom mg = make_geom(a.n, a.w, a.flags, x == 1);
+    p.h = mg.h;
+    p.causal = mg.causal; p.linear = mg.linear; p.one_sided = mg.one_sided;
+    p.full_range = mg.one_sided ? (a.w - 1 >= a.n) : (2ll * mg.h + 1 >= a.n);
+    p.n_tiles = (a.n + kTile - 1) / kTile;
+    p.scale = a.scale;
+    p.scale2 = a.scale * kLog2e;
+    for (int i = 0; i < 3; ++i) { p.qs[i] = a.qs[i]; p.ks[i] = a.ks[i]; }
+    const cudaError_t e = a.d == 128 ? launch_branch<128>(p, st) : launch_branch<64>(p, st);
+    if (e != cudaSuccess) return e;
+  }
+  return cudaSuccess;
+}
+
+}  // namespace sa
