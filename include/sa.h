@@ -114,13 +114,14 @@ sa_status sa_make_perm(uint64_t seed, uint32_t layer, int32_t B, int32_t n, int3
  * SA_STATIC_SCRATCH_BYTES that every GPU which loads the library holds until the process exits.
  *   - perm, inv: out, device, int32 [B,n], 16-byte aligned, owned by the caller as always.
  *   - Limit: sa_workspace_bytes(.., SA_OP_MAKE_PERM) for (B, n) must not exceed
- *     SA_STATIC_SCRATCH_BYTES (about 170,000 tokens in total, B*n); beyond that the call
+ *     SA_STATIC_SCRATCH_BYTES (about 200,000 tokens in total, B*n); beyond that the call
  *     returns SA_ERR_TOO_LARGE and launches nothing.
  *   - The call allocates and frees nothing, and only enqueues kernels on `stream`.
  *   - The first call on each device looks up the array's device address (one runtime query,
  *     with that device current); make that first call before starting any stream capture.
  *   - All calls on a device share the one array and it keeps whatever the last call left.
- *     No part of it has to be cleared: a call writes every word before reading it.  Two
+ *     The only part that must start at zero (the sort's bucket counters) is cleared by
+ *     each call on its stream; everything else is written before it is read.  Two
  *     calls whose kernels may run at the same time on one GPU (different streams, or
  *     different host threads) race on the array and give wrong permutations: keep the
  *     calls of a device on one stream, or order them yourself. */

@@ -192,7 +192,7 @@ def sa_make_perm_static(seed: int, layer: int, B: int, n: int, perm: torch.Tenso
     Same permutations as sa_make_perm, bit for bit.  The sort's scratch is a fixed array
     inside the library (STATIC_SCRATCH_BYTES per GPU), so this wrapper creates no tensor: the
     caller hands in both outputs (int32 [B,n], CUDA).  Raises SaError (status 7) when B*n
-    needs more scratch than is built in (roughly B*n > 170,000).  Calls that may overlap on
+    needs more scratch than is built in (roughly B*n > 200,000).  Calls that may overlap on
     one GPU race on the shared array: keep them on one stream."""
     lib = load_library()
     for t in (perm, inv):

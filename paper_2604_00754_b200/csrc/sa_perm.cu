@@ -1,21 +1,26 @@
-// Permutation generation (Alg. 1 line 1): Philox4x32-10 sort keys, a segmented
-// least-significant-digit radix sort (8 passes of 8 bits over 64-bit keys, one segment
-// per sequence), and the inverse by scatter, fused into the last pass.
-//
-// The radix sort is stable, so equal keys keep increasing token order: the result is
-// the unique ordering by (key, token).
+// Permutation generation (Alg. 1 line 1): Philox4x32-10 sort keys, a segmented sort by
+// (key, token) with one segment per sequence -- one radix pass on the leading key bits,
+// then ranking inside each bucket -- and the inverse written with the permutation.
 #include "sa_common.cuh"
 
 namespace sa {
 namespace {
 
-constexpr int kRadixBits = 8;
-constexpr int kRadix = 1 << kRadixBits;
-constexpr int kSortThreads = 256;
-constexpr int kSortWarps = kSortThreads / 32;
-constexpr int kItems = 8;                          // keys per thread per tile
-constexpr int kTile = kSortThreads * kItems;       // keys per block
-constexpr int kPasses = 64 / kRadixBits;
+// Sorting n 64-bit keys that are uniform random bits does not need eight radix passes:
+// one pass on the leading bits puts every key into a bucket of about 32 keys, and inside a
+// bucket the final place of a key is the number of bucket members that precede it in
+// (key, token) order, found by direct counting.  Four launches, no assumption on the bucket
+// sizes (an unlucky bucket only costs more comparisons), and the order inside a bucket after
+// the scatter does not matter, so the scatter may use atomics and the result is still the
+// unique ordering by (key, token).
+constexpr int kThreadsPerBlock = 256;
+constexpr int kMaxBucketBits = 16;
+
+__host__ __device__ inline int bucket_bits_for(int n) {
+  int bits = 0;
+  while (bits < kMaxBucketBits && (n >> (bits + 5)) > 0) ++bits;   // about 32 keys per bucket
+  return bits;
+}
 
 __device__ __forceinline__ void philox_round(uint32_t (&c)[4], uint32_t k0, uint32_t k1) {
   const uint32_t hi0 = __umulhi(0xD2511F53u, c[0]), lo0 = 0xD2511F53u * c[0];
@@ -37,112 +42,87 @@ __device__ __forceinline__ uint64_t sort_key(uint32_t seed_lo, uint32_t seed_hi,
   return ((uint64_t)c[0] << 32) | c[1];
 }
 
-__global__ void keys_kernel(uint32_t seed_lo, uint32_t seed_hi, uint32_t layer, int n,
-                            uint64_t* __restrict__ keys, int32_t* __restrict__ vals) {
+__device__ __forceinline__ uint32_t bucket_of(uint64_t key, int bits) {
+  return bits ? (uint32_t)(key >> (64 - bits)) : 0u;
+}
+
+// keys[b][i] and the size of every bucket.  counts must be zero on entry.
+__global__ void keys_kernel(uint32_t seed_lo, uint32_t seed_hi, uint32_t layer, int n, int bits,
+                            uint64_t* __restrict__ keys, uint32_t* __restrict__ counts) {
   const int b = blockIdx.y;
+  uint32_t* cb = counts + ((size_t)b << bits);
   for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
-    keys[(size_t)b * n + i] = sort_key(seed_lo, seed_hi, layer, b, i);
-    vals[(size_t)b * n + i] = i;
+    const uint64_t key = sort_key(seed_lo, seed_hi, layer, b, i);
+    keys[(size_t)b * n + i] = key;
+    atomicAdd(&cb[bucket_of(key, bits)], 1u);
   }
 }
 
-// counts[b][digit][blk] = number of keys of tile blk of sequence b with that digit.
-__global__ void __launch_bounds__(kSortThreads)
-hist_kernel(const uint64_t* __restrict__ keys, int n, int shift, int nblk,
-            uint32_t* __restrict__ counts) {
-  __shared__ uint32_t h[kRadix];
-  const int b = blockIdx.y, blk = blockIdx.x;
-  h[threadIdx.x] = 0;
-  __syncthreads();
-  const uint64_t* kb = keys + (size_t)b * n;
-  const int base = blk * kTile;
-#pragma unroll
-  for (int it = 0; it < kItems; ++it) {
-    const int i = base + it * kSortThreads + threadIdx.x;
-    if (i < n) atomicAdd(&h[(uint32_t)(kb[i] >> shift) & (kRadix - 1)], 1u);
-  }
-  __syncthreads();
-  counts[((size_t)b * kRadix + threadIdx.x) * nblk + blk] = h[threadIdx.x];
-}
-
-// Exclusive scan of counts[b][digit][blk] in (digit, blk) order, in place.  One block per b.
-__global__ void __launch_bounds__(kRadix)
-scan_kernel(uint32_t* __restrict__ counts, int nblk) {
-  __shared__ uint32_t tot[kRadix];
-  uint32_t* c = counts + (size_t)blockIdx.x * kRadix * nblk + (size_t)threadIdx.x * nblk;
+// Exclusive scan of the bucket sizes of one sequence, in place, and a copy that the
+// scatter advances.  One block per sequence.
+__global__ void __launch_bounds__(kThreadsPerBlock)
+scan_kernel(uint32_t* __restrict__ counts, uint32_t* __restrict__ cursor, int nbuckets) {
+  __shared__ uint32_t part[kThreadsPerBlock];
+  uint32_t* c = counts + (size_t)blockIdx.x * nbuckets;
+  uint32_t* cur = cursor + (size_t)blockIdx.x * nbuckets;
+  const int per = (nbuckets + kThreadsPerBlock - 1) / kThreadsPerBlock;
+  const int lo = threadIdx.x * per, hi = min(lo + per, nbuckets);
   uint32_t s = 0;
-  for (int j = 0; j < nblk; ++j) s += c[j];
-  tot[threadIdx.x] = s;
+  for (int j = lo; j < hi; ++j) s += c[j];
+  part[threadIdx.x] = s;
   __syncthreads();
-  // Hillis-Steele inclusive scan over the 256 digit totals
-  for (int o = 1; o < kRadix; o <<= 1) {
-    const uint32_t add = threadIdx.x >= o ? tot[threadIdx.x - o] : 0u;
+  for (int o = 1; o < kThreadsPerBlock; o <<= 1) {
+    const uint32_t add = threadIdx.x >= o ? part[threadIdx.x - o] : 0u;
     __syncthreads();
-    tot[threadIdx.x] += add;
+    part[threadIdx.x] += add;
     __syncthreads();
   }
-  uint32_t run = tot[threadIdx.x] - s;  // exclusive start of this digit
-  for (int j = 0; j < nblk; ++j) {
+  uint32_t run = part[threadIdx.x] - s;
+  for (int j = lo; j < hi; ++j) {
     const uint32_t v = c[j];
     c[j] = run;
+    cur[j] = run;
     run += v;
   }
 }
 
-// Stable scatter of one tile.  Keys are taken 256 at a time in index order; inside a
-// group, a key's rank among equal digits is (equal digits in earlier warps) + (equal
-// digits in lower lanes of its own warp).  With `last`, the sorted token list IS perm and
-// the inverse is written in the same pass.
-__global__ void __launch_bounds__(kSortThreads)
-scatter_kernel(const uint64_t* __restrict__ keys_in, const int32_t* __restrict__ vals_in,
-               uint64_t* __restrict__ keys_out, int32_t* __restrict__ vals_out,
-               int32_t* __restrict__ inv_out, int n, int shift, int nblk,
-               const uint32_t* __restrict__ offsets, int last) {
-  __shared__ uint32_t base[kRadix];
-  __shared__ uint32_t whist[kSortWarps][kRadix];
-  const int b = blockIdx.y, blk = blockIdx.x;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  base[threadIdx.x] = offsets[((size_t)b * kRadix + threadIdx.x) * nblk + blk];
-  const uint64_t* kb = keys_in + (size_t)b * n;
-  const int32_t* vb = vals_in + (size_t)b * n;
-  for (int it = 0; it < kItems; ++it) {
-    for (int x = threadIdx.x; x < kSortWarps * kRadix; x += kSortThreads) (&whist[0][0])[x] = 0;
-    __syncthreads();
-    const int i = blk * kTile + it * kSortThreads + threadIdx.x;
-    const bool live = i < n;
-    uint64_t key = 0;
-    int32_t val = 0;
-    uint32_t digit = 0, rank = 0;
-    if (live) { key = kb[i]; val = vb[i]; digit = (uint32_t)(key >> shift) & (kRadix - 1); }
-    // dead lanes get a private pseudo-digit so they never match a live one
-    const uint32_t peers = __match_any_sync(0xffffffffu, live ? digit : (kRadix + lane));
-    if (live) {
-      rank = __popc(peers & ((1u << lane) - 1u));
-      if (rank == 0) whist[warp][digit] = __popc(peers);
+// Every (key, token) into its bucket's range, in arbitrary order inside the range.
+__global__ void scatter_kernel(const uint64_t* __restrict__ keys, uint32_t* __restrict__ cursor,
+                               uint64_t* __restrict__ bkeys, int32_t* __restrict__ btoks, int n,
+                               int bits) {
+  const int b = blockIdx.y;
+  uint32_t* cur = cursor + ((size_t)b << bits);
+  for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+    const uint64_t key = keys[(size_t)b * n + i];
+    const uint32_t pos = atomicAdd(&cur[bucket_of(key, bits)], 1u);
+    bkeys[(size_t)b * n + pos] = key;
+    btoks[(size_t)b * n + pos] = i;
+  }
+}
+
+// Slot of every token: start of its bucket plus the number of bucket members that come
+// first in (key, token) order.  Writes perm and its inverse.
+__global__ void rank_kernel(const uint64_t* __restrict__ bkeys, const int32_t* __restrict__ btoks,
+                            const uint32_t* __restrict__ starts, int32_t* __restrict__ perm,
+                            int32_t* __restrict__ inv, int n, int bits) {
+  const int b = blockIdx.y;
+  const uint64_t* kb = bkeys + (size_t)b * n;
+  const int32_t* tb = btoks + (size_t)b * n;
+  const uint32_t* st = starts + ((size_t)b << bits);
+  const uint32_t nbuckets = 1u << bits;
+  for (int e = blockIdx.x * blockDim.x + threadIdx.x; e < n; e += gridDim.x * blockDim.x) {
+    const uint64_t key = kb[e];
+    const int32_t tok = tb[e];
+    const uint32_t bk = bucket_of(key, bits);
+    const uint32_t lo = st[bk], hi = bk + 1 < nbuckets ? st[bk + 1] : (uint32_t)n;
+    uint32_t rank = 0;
+    for (uint32_t j = lo; j < hi; ++j) {
+      const uint64_t kj = kb[j];
+      rank += (kj < key) || (kj == key && tb[j] < tok);
     }
-    __syncthreads();
-    uint32_t pos = 0;
-    if (live) {
-      pos = base[digit] + rank;
-      for (int wv = 0; wv < warp; ++wv) pos += whist[wv][digit];
-    }
-    __syncthreads();
-    {  // advance the running base of digit threadIdx.x past this group
-      uint32_t add = 0;
-#pragma unroll
-      for (int wv = 0; wv < kSortWarps; ++wv) add += whist[wv][threadIdx.x];
-      base[threadIdx.x] += add;
-    }
-    if (live) {
-      if (last) {
-        vals_out[(size_t)b * n + pos] = val;
-        inv_out[(size_t)b * n + val] = (int32_t)pos;
-      } else {
-        keys_out[(size_t)b * n + pos] = key;
-        vals_out[(size_t)b * n + pos] = val;
-      }
-    }
-    __syncthreads();
+    const int32_t pos = (int32_t)(lo + rank);
+    perm[(size_t)b * n + pos] = tok;
+    inv[(size_t)b * n + tok] = pos;
   }
 }
 
@@ -182,40 +162,31 @@ unsigned char* static_scratch_ptr() {
 
 size_t make_perm_ws_bytes(int B, int n) {
   const size_t bn = (size_t)B * n;
-  const int nblk = (n + kTile - 1) / kTile;
-  return 2 * align_up(bn * 8, 256) + 2 * align_up(bn * 4, 256) +
-         align_up((size_t)B * kRadix * nblk * 4, 256);
+  const size_t nb = (size_t)B << bucket_bits_for(n);
+  return 2 * align_up(bn * 8, 256) + align_up(bn * 4, 256) + 2 * align_up(nb * 4, 256);
 }
 
 cudaError_t launch_make_perm(uint64_t seed, uint32_t layer, int B, int n, int32_t* perm,
                              int32_t* inv, void* ws, cudaStream_t st) {
   const size_t bn = (size_t)B * n;
-  const int nblk = (n + kTile - 1) / kTile;
+  const int bits = bucket_bits_for(n);
+  const size_t nb = (size_t)B << bits;
   char* p = (char*)ws;
-  uint64_t* keys[2];
-  int32_t* vals[2];
-  keys[0] = (uint64_t*)p; p += align_up(bn * 8, 256);
-  keys[1] = (uint64_t*)p; p += align_up(bn * 8, 256);
-  vals[0] = (int32_t*)p; p += align_up(bn * 4, 256);
-  vals[1] = (int32_t*)p; p += align_up(bn * 4, 256);
-  uint32_t* counts = (uint32_t*)p;
+  uint64_t* keys = (uint64_t*)p; p += align_up(bn * 8, 256);
+  uint64_t* bkeys = (uint64_t*)p; p += align_up(bn * 8, 256);
+  int32_t* btoks = (int32_t*)p; p += align_up(bn * 4, 256);
+  uint32_t* counts = (uint32_t*)p; p += align_up(nb * 4, 256);
+  uint32_t* cursor = (uint32_t*)p;
 
-  const int kb = min((n + 255) / 256, 1024);
-  keys_kernel<<<dim3(kb, B), 256, 0, st>>>((uint32_t)seed, (uint32_t)(seed >> 32), layer, n,
-                                           keys[0], vals[0]);
-  bump_launches();
-  int cur = 0;
-  for (int pass = 0; pass < kPasses; ++pass) {
-    const int shift = pass * kRadixBits;
-    const int last = pass == kPasses - 1;
-    hist_kernel<<<dim3(nblk, B), kSortThreads, 0, st>>>(keys[cur], n, shift, nblk, counts);
-    scan_kernel<<<B, kRadix, 0, st>>>(counts, nblk);
-    scatter_kernel<<<dim3(nblk, B), kSortThreads, 0, st>>>(
-        keys[cur], vals[cur], keys[cur ^ 1], last ? perm : vals[cur ^ 1], inv, n, shift, nblk,
-        counts, last);
-    bump_launches(3);
-    cur ^= 1;
-  }
+  cudaError_t e = cudaMemsetAsync(counts, 0, nb * 4, st);   // bucket sizes start at zero
+  if (e != cudaSuccess) return e;
+  const int kb = min((n + kThreadsPerBlock - 1) / kThreadsPerBlock, 1024);
+  keys_kernel<<<dim3(kb, B), kThreadsPerBlock, 0, st>>>((uint32_t)seed, (uint32_t)(seed >> 32),
+                                                        layer, n, bits, keys, counts);
+  scan_kernel<<<B, kThreadsPerBlock, 0, st>>>(counts, cursor, 1 << bits);
+  scatter_kernel<<<dim3(kb, B), kThreadsPerBlock, 0, st>>>(keys, cursor, bkeys, btoks, n, bits);
+  rank_kernel<<<dim3(kb, B), kThreadsPerBlock, 0, st>>>(bkeys, btoks, counts, perm, inv, n, bits);
+  bump_launches(4);
   return cudaGetLastError();
 }
 
@@ -240,9 +211,9 @@ extern "C" sa_status sa_make_perm_static(uint64_t seed, uint32_t layer, int32_t 
   if (make_perm_ws_bytes(B, n) > (size_t)SA_STATIC_SCRATCH_BYTES) return SA_ERR_TOO_LARGE;
   unsigned char* scratch = static_scratch_ptr();
   if (!scratch) return SA_ERR_CUDA;
-  // Nothing in the scratch has to start at zero: the key, index and histogram arrays of a
-  // call are each written in full by that call before anything reads them, so whatever
-  // the previous call left behind is never seen.
+  // Only the bucket counters have to start at zero, and the launcher clears them on the
+  // stream itself; the key and token arrays are written in full before anything reads
+  // them, so whatever the previous call left behind is never seen.
   return launch_make_perm(seed, layer, B, n, perm, inv, scratch, (cudaStream_t)stream) ==
                  cudaSuccess ? SA_OK : SA_ERR_CUDA;
 }
