@@ -496,7 +496,9 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
         const int cls = tile_class(p, q0, kv, kHalf);
         const int hb = h & 1;
         const uint32_t tg = gt0 + (h >> 1);
-        ok = mbar_wait(bar(C::kBarTokFull + tg % C::kTok), (tg / C::kTok) & 1u, gave_up, p.status);
+        // the token list belongs to the whole 128-key tile: wait for it at its first half only
+        if (hb == 0 || h == cur.first)
+          ok = mbar_wait(bar(C::kBarTokFull + tg % C::kTok), (tg / C::kTok) & 1u, gave_up, p.status);
         if (ok)
           ok = mbar_wait(bar(C::kBarSFull + 2 * t + hb), (hb ? s_cnt1 : s_cnt0) & 1u, gave_up,
                          p.status);

@@ -76,6 +76,10 @@ SMALL = [
     (1, 6, 2, 511, 128, 129, CAUSAL),
     (1, 1, 1, 700, 256, 40, 0),
     (1, 3, 3, 64, 8, 5, LINEAR_WINDOW),
+    (2, 3, 3, 1000, 64, 300, CAUSAL),                   # odd group size: two slot tiles per item
+    (1, 8, 2, 1153, 64, 128, CAUSAL),                   # w = tile width, ragged tail, GQA
+    (1, 4, 4, 640, 128, 1, 0),                          # w = 1 on the tensor-core path
+    (1, 2, 1, 900, 128, 257, LINEAR_WINDOW),
 ]
 
 
@@ -266,6 +270,10 @@ def run_backward(q, k, v, dy, lg, perm, inv, w, flags):
     (1, 2, 2, 130, 128, 40, 0),
     (1, 2, 1, 77, 32, 300, CAUSAL),
     (1, 1, 1, 260, 64, 1, CAUSAL | SWA_ONE_SIDED),
+    (1, 8, 2, 700, 128, 200, CAUSAL | SWA_ONE_SIDED),   # GQA group of 4, several tiles, wrap-around
+    (2, 2, 1, 515, 64, 129, CAUSAL | LINEAR_WINDOW),    # no wrap, ragged last tile
+    (1, 2, 2, 384, 128, 96, 0),                         # non-causal, n a tile multiple
+    (1, 2, 1, 200, 64, 1000, CAUSAL | SWA_ONE_SIDED),   # w > n: every causal key, two tiles
 ])
 def test_backward_small(B, Hq, Hkv, n, d, w, flags, gated, dtype):
     q, k, v = draw((B, Hq, n, d), (B, Hkv, n, d), dtype, seed=n)
