@@ -32,7 +32,6 @@ namespace {
 
 constexpr int kTile = 128;           // query rows per tile and keys per K/V tile
 constexpr int kThreads = 384;
-constexpr int kHalf = 64;            // keys per score block (half a K/V tile)
 constexpr int kProducers = 96;       // threads of the three gather warps
 constexpr uint32_t kTmemCols = 512;
 
@@ -89,17 +88,17 @@ __device__ __forceinline__ int tile_class(const TcParams& p, int q0, int kv, int
   return kCausalOnly;
 }
 
-// The half-steps h (keys kstart + 64 h ... + 63) that tile_class does not skip for the
+// The score blocks h (keys kstart + (h << shift) and the 2^shift - 1 after it) that tile_class does not skip for the
 // query tile at q0: a contiguous range [first, last], empty (first > last) for a tile
 // that does not exist.
 __device__ __forceinline__ void active_halves(const TcParams& p, int q0, int valid, int kstart,
-                                              int H, int* first, int* last) {
+                                              int H, int shift, int* first, int* last) {
   const int q1 = q0 + kTile - 1;
   int lo, hi;   // keys of interest: some key of the half >= lo, its first key <= hi
   if (p.full_range) { lo = 0; hi = p.n - 1; }
   else if (p.one_sided) { lo = q0 - (p.w - 1); hi = q1; }
   else { lo = q0 - p.h; hi = q1 + p.h; }
-  const int f = max(0, (lo - kstart) >> 6), l = min(H - 1, (hi - kstart) >> 6);
+  const int f = max(0, (lo - kstart) >> shift), l = min(H - 1, (hi - kstart) >> shift);
   *first = valid ? f : (1 << 30);
   *last = valid ? l : -1;
 }
@@ -183,10 +182,16 @@ struct Cfg {
 
 // ------------------------------------------------------------------------- kernel
 
-template <int D>
+// D: head dimension.  KB: keys per score block, 64 or 128.  With 64 a tile's S columns hold
+// two blocks and the scores run two blocks ahead of the softmax; with 128 a block is the
+// whole K/V tile and the next scores of a tile follow its P V.
+template <int D, int KB>
 __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_constant__ TcParams p) {
   extern __shared__ __align__(1024) uint8_t smem[];
   using C = Cfg<D>;
+  constexpr int kHalf = KB;             // keys per score block
+  constexpr int NB = kTile / KB;        // score blocks per K/V tile = S buffers per query tile
+  constexpr int kShift = KB == 64 ? 6 : 7;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (p.abort_flag && *p.abort_flag) return;  // an earlier check rejected perm/inv (uniform)
@@ -375,17 +380,19 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
       auto issue_pv = [&](int t, int b, uint32_t v_lo, uint32_t acc0) {
         const uint64_t vd = desc64((v_lo + b * (kHalf * 128 >> 4)) | kLoV, kDescHi);
         mma_ts_x4(tmem + C::kColO + t * D, tmem + t * 128 + b * kHalf, vd, idesc_pv, acc0);
+        if (KB == 128)
+          mma_ts_x4(tmem + C::kColO + t * D, tmem + t * 128 + 32, vd + 512, idesc_pv, 1u);
         tc_commit(bar(C::kBarPvDone + t));
       };
       for (int w_item = blockIdx.x; w_item < p.total_items && ok; w_item += gridDim.x, ++it) {
         const int item = w_item % p.items_per_kv, bh = w_item / p.items_per_kv;
         const Geo g = make_geo(p, item, bh % p.Hkv);
-        const int H = 2 * g.T;          // half-steps of this item
+        const int H = NB * g.T;         // score blocks of this item
         // half-steps [first, last] that each query tile takes part in (a contiguous range);
         // everything per tile is kept in scalars so that nothing is indexed at run time
         int first0, first1, last0, last1;
-        active_halves(p, g.q0[0], g.valid[0], g.kstart, H, &first0, &last0);
-        active_halves(p, g.q0[1], g.valid[1], g.kstart, H, &first1, &last1);
+        active_halves(p, g.q0[0], g.valid[0], g.kstart, H, kShift, &first0, &last0);
+        active_halves(p, g.q0[1], g.valid[1], g.kstart, H, kShift, &first1, &last1);
         uint32_t started0 = 0, started1 = 0;
         // ring uses of this item: K_j = use + 2j, V_j = use + 2j + 1
         ok = mbar_wait(bar(C::kBarQFull), it & 1u, gave_up, p.status);
@@ -397,8 +404,10 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
           const uint32_t k0 = slot_lo(use);
           if (first0 <= 0 && last0 >= 0) issue_qk(0, 0, k0);
           if (first1 <= 0 && last1 >= 0) issue_qk(1, 0, k0);
-          if (first0 <= 1 && last0 >= 1) issue_qk(0, 1, k0);
-          if (first1 <= 1 && last1 >= 1) issue_qk(1, 1, k0);
+          if (NB == 2) {
+            if (first0 <= 1 && last0 >= 1) issue_qk(0, 1, k0);
+            if (first1 <= 1 && last1 >= 1) issue_qk(1, 1, k0);
+          }
         }
         tc_commit(bar(C::kBarSlotEmpty + use % C::kSlots));
         if (g.T == 1) tc_commit(bar(C::kBarQEmpty));
@@ -414,7 +423,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
           // one (tile, half) unit: P V of half-step h, then Q K^T of half-step h + 2
           auto unit = [&](auto tc, auto bc, int first, int last, uint32_t& started, uint32_t& pcnt) {
             constexpr int t = decltype(tc)::value, b = decltype(bc)::value;
-            const int h = 2 * j + b;
+            const int h = NB * j + b;
             if (h >= first && h <= last) {
               ok = mbar_wait(bar(C::kBarPReady + 2 * t + b), pcnt & 1u, gave_up, p.status);
               if (!ok) return;
@@ -424,14 +433,16 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
               started = 1;
               if (h == last) tc_commit(bar(C::kBarODone + t));
             }
-            if (more && h + 2 >= first && h + 2 <= last) issue_qk(t, b, k_lo);
+            if (more && h + NB >= first && h + NB <= last) issue_qk(t, b, k_lo);
           };
           using I0 = std::integral_constant<int, 0>;
           using I1 = std::integral_constant<int, 1>;
           unit(I0{}, I0{}, first0, last0, started0, pc00);
           if (ok) unit(I1{}, I0{}, first1, last1, started1, pc10);
-          if (ok) unit(I0{}, I1{}, first0, last0, started0, pc01);
-          if (ok) unit(I1{}, I1{}, first1, last1, started1, pc11);
+          if (NB == 2) {
+            if (ok) unit(I0{}, I1{}, first0, last0, started0, pc01);
+            if (ok) unit(I1{}, I1{}, first1, last1, started1, pc11);
+          }
           if (!ok) break;
           // the slots free when the products issued so far have finished
           tc_commit(bar(C::kBarSlotEmpty + uv % C::kSlots));
@@ -466,7 +477,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
       c.valid = t ? g.valid[1] : g.valid[0];
       c.kstart = g.kstart;
       c.T = g.T;
-      active_halves(p, c.q0, c.valid, c.kstart, 2 * c.T, &c.first, &c.last);
+      active_halves(p, c.q0, c.valid, c.kstart, NB * c.T, kShift, &c.first, &c.last);
       const int qv = c.q0 + row;
       c.row_valid = c.valid && qv < p.n;
       c.q_tok = c.row_valid ? (p.perm ? p.perm[(size_t)c.b * p.n + qv] : qv) : 0;
@@ -494,8 +505,8 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
       for (int h = cur.first; h <= cur.last; ++h) {
         const int kv = cur.kstart + h * kHalf;
         const int cls = tile_class(p, q0, kv, kHalf);
-        const int hb = h & 1;
-        const uint32_t tg = gt0 + (h >> 1);
+        const int hb = h & (NB - 1);
+        const uint32_t tg = gt0 + (h >> (NB - 1));
         // the token list belongs to the whole 128-key tile: wait for it at its first half only
         if (hb == 0 || h == cur.first)
           ok = mbar_wait(bar(C::kBarTokFull + tg % C::kTok), (tg / C::kTok) & 1u, gave_up, p.status);
@@ -580,7 +591,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
         const float neg = (m == -INFINITY) ? 0.f : -m * p.scale2;
         const float2 sc2 = make_float2(p.scale2, p.scale2), ng2 = make_float2(neg, neg);
         float2 lsum = make_float2(0.f, 0.f);
-        uint32_t pk[kHalf / 2];
+        uint32_t pk[kHalf / 2];   // two bf16 per word
 #pragma unroll
         for (int x = 0; x < kHalf / 2; ++x) {
           const float2 a = __ffma2_rn(make_float2(__uint_as_float(sr[2 * x]),
@@ -590,7 +601,9 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
           const __nv_bfloat162 h2 = __floats2bfloat162_rn(e.x, e.y);
           pk[x] = *reinterpret_cast<const uint32_t*>(&h2);
         }
-        tmem_st32(sh_addr, pk);
+#pragma unroll
+        for (int c = 0; c < kHalf / 64; ++c)
+          tmem_st32(sh_addr + 32 * c, reinterpret_cast<const uint32_t(&)[32]>(pk[32 * c]));
         l += lsum.x + lsum.y;
         tmem_wait_st();
         tc_fence_before();
@@ -682,6 +695,18 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
 
 // ---------------------------------------------------------------------------- host
 
+// Score-block width.  Narrow windows skip more with 64-key blocks; from w = 256 on the
+// 128-key block wins (half as many products, commits and softmax rounds per key).  The
+// environment variable SA_KEY_BLOCK=64|128 overrides the choice so tests can run both.
+bool key_block_128(int w) {
+  static int forced = -1;
+  if (forced < 0) {
+    const char* e = getenv("SA_KEY_BLOCK");
+    forced = !e ? 0 : (e[0] == '6' ? 64 : 128);
+  }
+  return forced ? forced == 128 : w > 128;
+}
+
 bool tc_disabled() {
   static int v = -1;
   if (v < 0) {
@@ -729,17 +754,18 @@ cudaError_t launch_fwd_tc(const FwdArgs& a, cudaStream_t st) {
     if (e != cudaSuccess) return e;
   }
   const unsigned grid = (unsigned)min(p.total_items, sm_count[dev]);
-  if (a.d == 128) {
-    const int smem = Cfg<128>::kBytes;
-    e = cudaFuncSetAttribute(fwd_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return e;
-    fwd_tc_kernel<128><<<grid, kThreads, smem, st>>>(p);
-  } else {
-    const int smem = Cfg<64>::kBytes;
-    e = cudaFuncSetAttribute(fwd_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e != cudaSuccess) return e;
-    fwd_tc_kernel<64><<<grid, kThreads, smem, st>>>(p);
-  }
+  const bool wide = key_block_128(a.w);
+  auto go = [&](auto kernel, int smem) {
+    cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (err != cudaSuccess) return err;
+    kernel<<<grid, kThreads, smem, st>>>(p);
+    return cudaSuccess;
+  };
+  if (a.d == 128)
+    e = wide ? go(fwd_tc_kernel<128, 128>, Cfg<128>::kBytes) : go(fwd_tc_kernel<128, 64>, Cfg<128>::kBytes);
+  else
+    e = wide ? go(fwd_tc_kernel<64, 128>, Cfg<64>::kBytes) : go(fwd_tc_kernel<64, 64>, Cfg<64>::kBytes);
+  if (e != cudaSuccess) return e;
   bump_launches();
   return cudaGetLastError();
 }

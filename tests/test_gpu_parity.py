@@ -113,6 +113,18 @@ def test_swa_forward_small(B, Hq, Hkv, n, d, w, flags, dtype):
     assert np.abs(as_f64(lse) - rlse).max() <= (1e-4 if dtype == torch.float32 else 2e-2)
 
 
+@pytest.mark.parametrize("block", ["64", "128"])
+def test_both_score_block_widths(block):
+    # the tensor-core forward has a 64-key and a 128-key score block; the library picks by w,
+    # a child process with SA_KEY_BLOCK set runs the other one on the same cases
+    import os, subprocess, sys
+    env = dict(os.environ, SA_KEY_BLOCK=block)
+    r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-m", "gpu", __file__, "-k",
+                        "test_sa_forward_small or test_swa_forward_small or test_gated_forward_small"],
+                       env=env, capture_output=True, text=True)
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+
+
 def test_identity_permutation_equals_swa_on_device():
     B, Hq, Hkv, n, d, w = 1, 2, 1, 333, 64, 17
     q, k, v = draw((B, Hq, n, d), (B, Hkv, n, d), torch.float32, seed=1)
