@@ -591,19 +591,21 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
         const float neg = (m == -INFINITY) ? 0.f : -m * p.scale2;
         const float2 sc2 = make_float2(p.scale2, p.scale2), ng2 = make_float2(neg, neg);
         float2 lsum = make_float2(0.f, 0.f);
-        uint32_t pk[kHalf / 2];   // two bf16 per word
 #pragma unroll
-        for (int x = 0; x < kHalf / 2; ++x) {
-          const float2 a = __ffma2_rn(make_float2(__uint_as_float(sr[2 * x]),
-                                                  __uint_as_float(sr[2 * x + 1])), sc2, ng2);
-          const float2 e = make_float2(exp2f(a.x), exp2f(a.y));
-          lsum = __fadd2_rn(lsum, e);
-          const __nv_bfloat162 h2 = __floats2bfloat162_rn(e.x, e.y);
-          pk[x] = *reinterpret_cast<const uint32_t*>(&h2);
+        for (int c = 0; c < kHalf / 64; ++c) {
+          uint32_t pk[32];          // 64 probabilities, two bf16 per word
+#pragma unroll
+          for (int x = 0; x < 32; ++x) {
+            const float2 a = __ffma2_rn(make_float2(__uint_as_float(sr[64 * c + 2 * x]),
+                                                    __uint_as_float(sr[64 * c + 2 * x + 1])),
+                                        sc2, ng2);
+            const float2 e = make_float2(exp2f(a.x), exp2f(a.y));
+            lsum = __fadd2_rn(lsum, e);
+            const __nv_bfloat162 h2 = __floats2bfloat162_rn(e.x, e.y);
+            pk[x] = *reinterpret_cast<const uint32_t*>(&h2);
+          }
+          tmem_st32(sh_addr + 32 * c, pk);
         }
-#pragma unroll
-        for (int c = 0; c < kHalf / 64; ++c)
-          tmem_st32(sh_addr + 32 * c, reinterpret_cast<const uint32_t(&)[32]>(pk[32 * c]));
         l += lsum.x + lsum.y;
         tmem_wait_st();
         tc_fence_before();
