@@ -18,6 +18,10 @@
 // Rows of every operand are gathered through perm with cp.async into swizzled shared
 // memory, as in the forward kernel; finished rows are scattered to their original places.
 //
+// The column tile is 128 or 64 wide (template KC).  64 halves the band-edge waste of narrow
+// windows and, where scores and accumulators then fit in 256 tensor-memory columns, lets two
+// CTAs share an SM so that one CTA's loads and epilogue hide behind the other's products.
+//
 // Warp roles (256 threads): warp 0 MMA issuer and TMEM allocator, warps 1-3 gather
 // producers, warps 4-7 one thread per row.  Every mbarrier wait is bounded.
 #include "sa_bwd_tc.cuh"
@@ -29,7 +33,6 @@ namespace {
 constexpr int kTile = 128;
 constexpr int kBwdThreads = 256;
 constexpr int kProducers = 96;
-constexpr uint32_t kTmemCols = 512;
 
 struct BwdTcParams {
   const void *q, *k, *v, *dy;
@@ -51,7 +54,7 @@ struct BwdTcParams {
 // Columns (virtual slots) a row tile starting at slot r0 has to meet: [cstart, cend].
 // rows_are_keys selects the transposed window of the one-sided rule.
 __device__ __forceinline__ void column_range(const BwdTcParams& p, int r0, bool rows_are_keys,
-                                             int* cstart, int* T) {
+                                             int kc, int* cstart, int* T) {
   const int rl = min(r0 + kTile - 1, p.n - 1);
   int lo, hi;
   if (p.full_range) { lo = 0; hi = p.n - 1; }
@@ -61,7 +64,7 @@ __device__ __forceinline__ void column_range(const BwdTcParams& p, int r0, bool 
   } else if (p.linear) { lo = max(r0 - p.h, 0); hi = min(rl + p.h, p.n - 1); }
   else { lo = r0 - p.h; hi = rl + p.h; }
   *cstart = lo;
-  *T = (hi - lo + kTile) / kTile;
+  *T = (hi - lo + kc) / kc;
 }
 
 __device__ __forceinline__ int actual_slot(const BwdTcParams& p, int v) {
@@ -70,14 +73,16 @@ __device__ __forceinline__ int actual_slot(const BwdTcParams& p, int v) {
   return v < 0 ? v + p.n : v;
 }
 
-template <int D>
+template <int D, int KC, int MODE>
 struct BCfg {
-  static constexpr int kTileBytes = kTile * D * 2;
-  static constexpr int kChunkBytes = kTile * 128;
+  static constexpr int kTileBytes = kTile * D * 2;              // a row-operand tile
+  static constexpr int kChunkBytes = kTile * 128;               // its 64-column blocks
+  static constexpr int kColBytes = KC * D * 2;                  // a column tile
+  static constexpr int kColChunkBytes = KC * 128;
   static constexpr int kStages = 2;
   static constexpr int kOffR = 0;                               // two row-operand tiles
   static constexpr int kOffC = 2 * kTileBytes;                  // kStages x two column tiles
-  static constexpr int kOffRowTok = kOffC + kStages * 2 * kTileBytes;
+  static constexpr int kOffRowTok = kOffC + kStages * 2 * kColBytes;
   static constexpr int kOffColTok = kOffRowTok + kTile * 4;     // kStages x 128 ints
   static constexpr int kOffColVec = kOffColTok + kStages * kTile * 4;  // kStages x 2 x 128 floats
   static constexpr int kOffBar = kOffColVec + kStages * 2 * kTile * 4;
@@ -87,16 +92,21 @@ struct BCfg {
                        kNumBars = kBarODone + 1;
   static constexpr int kOffMisc = kOffBar + kNumBars * 8;
   static constexpr int kBytes = kOffMisc + 16;
-  // tensor memory columns: S and dS at 0, dP and P at 128, accumulators from 256
-  static constexpr uint32_t kColS = 0, kColP = 128, kColAcc = 256;
+  // tensor memory columns: S and dS at 0, dP and P at KC, accumulators from 2 KC
+  static constexpr uint32_t kColS = 0, kColP = KC, kColAcc = 2 * KC;
+  static constexpr uint32_t kColsUsed = 2 * KC + (MODE == 1 ? 2 : 1) * D;
+  static constexpr uint32_t kTmemCols = kColsUsed <= 256 ? 256 : 512;
+  static constexpr int kCtasPerSm = (kTmemCols == 256 && kBytes <= 110 * 1024) ? 2 : 1;
   static_assert(kBytes <= 232448, "shared memory");
 };
 
 // MODE 0: rows are queries (dQ).  MODE 1: rows are keys (dK, dV).
-template <int D, int MODE>
-__global__ void __launch_bounds__(kBwdThreads, 1) bwd_tc_kernel(const __grid_constant__ BwdTcParams p) {
+template <int D, int KC, int MODE>
+__global__ void __launch_bounds__(kBwdThreads, BCfg<D, KC, MODE>::kCtasPerSm)
+bwd_tc_kernel(const __grid_constant__ BwdTcParams p) {
   extern __shared__ __align__(1024) uint8_t smem[];
-  using C = BCfg<D>;
+  using C = BCfg<D, KC, MODE>;
+  constexpr uint32_t kTmemCols = C::kTmemCols;
   constexpr bool kKeys = MODE == 1;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -119,7 +129,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_tc_kernel(const __grid_con
   const int hk = kKeys ? hr : hr / p.G;
   const int r0 = tile * kTile;
   int cstart, T;
-  column_range(p, r0, kKeys, &cstart, &T);
+  column_range(p, r0, kKeys, KC, &cstart, &T);
   const int iters = kKeys ? T * p.G : T;      // column tiles (times query heads of the group)
   const int32_t* perm = p.perm ? p.perm + (size_t)b * p.n : nullptr;
 
@@ -147,7 +157,6 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_tc_kernel(const __grid_con
     constexpr int kRpi = 32 / kCpr;        // rows per warp instruction
     const int ptid = threadIdx.x - 32;     // 0..95
     const int sub = lane / kCpr, chunk = lane % kCpr;
-    const uint32_t dst_lane = (uint32_t)(chunk >> 3) * C::kChunkBytes;
     const __nv_bfloat16* qg = (const __nv_bfloat16*)p.q;
     const __nv_bfloat16* kg = (const __nv_bfloat16*)p.k;
     const __nv_bfloat16* vg = (const __nv_bfloat16*)p.v;
@@ -156,13 +165,15 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_tc_kernel(const __grid_con
     auto signal = [&](uint32_t mb) {
       asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(mb) : "memory");
     };
+    // rows x D elements into a tile whose 64-column blocks are rows x 128 bytes each
     auto gather = [&](const __nv_bfloat16* base, int64_t tok_stride, const int32_t* toks,
-                      uint32_t dst_tile) {
+                      uint32_t dst_tile, int rows) {
 #pragma unroll 4
-      for (int grp = warp - 1; grp < kTile / kRpi; grp += 3) {
+      for (int grp = warp - 1; grp < rows / kRpi; grp += 3) {
         const int r = grp * kRpi + sub;
         const __nv_bfloat16* src = base + (int64_t)toks[r] * tok_stride + chunk * 8;
-        const uint32_t dst = dst_tile + dst_lane + r * 128 + (((chunk & 7) ^ (r & 7)) << 4);
+        const uint32_t dst = dst_tile + (uint32_t)(chunk >> 3) * (rows * 128) + r * 128 +
+                             (((chunk & 7) ^ (r & 7)) << 4);
         asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
       }
     };
@@ -188,11 +199,11 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_tc_kernel(const __grid_con
     bool live = !group_sync_stop();
     if (live) {
       if (kKeys) {
-        gather(kg + b * p.ks[0] + hr * p.ks[1], p.ks[2], rowtok, sbase + C::kOffR);
-        gather(vg + b * p.ks[0] + hr * p.ks[1], p.ks[2], rowtok, sbase + C::kOffR + C::kTileBytes);
+        gather(kg + b * p.ks[0] + hr * p.ks[1], p.ks[2], rowtok, sbase + C::kOffR, kTile);
+        gather(vg + b * p.ks[0] + hr * p.ks[1], p.ks[2], rowtok, sbase + C::kOffR + C::kTileBytes, kTile);
       } else {
-        gather(qg + b * p.qs[0] + hr * p.qs[1], p.qs[2], rowtok, sbase + C::kOffR);
-        gather(dyg + b * p.qs[0] + hr * p.qs[1], p.qs[2], rowtok, sbase + C::kOffR + C::kTileBytes);
+        gather(qg + b * p.qs[0] + hr * p.qs[1], p.qs[2], rowtok, sbase + C::kOffR, kTile);
+        gather(dyg + b * p.qs[0] + hr * p.qs[1], p.qs[2], rowtok, sbase + C::kOffR + C::kTileBytes, kTile);
       }
       signal(bar(C::kBarRFull));
     }
@@ -204,31 +215,35 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_tc_kernel(const __grid_con
         mbar_wait(bar(C::kBarCEmpty + s), ((it >> 1) - 1) & 1u, gave_up, p.status);
       int32_t* coltok = reinterpret_cast<int32_t*>(smem + C::kOffColTok) + s * kTile;
       const uint32_t colvec = sbase + C::kOffColVec + s * 2 * kTile * 4;
-      const int t0 = tok_of(actual_slot(p, cstart + j * kTile + ptid));
-      coltok[ptid] = t0;
-      int t1 = 0;
-      if (ptid < 32) {
-        t1 = tok_of(actual_slot(p, cstart + j * kTile + ptid + 96));
+      int t0 = 0, t1 = 0;
+      if (ptid < KC) {
+        t0 = tok_of(actual_slot(p, cstart + j * KC + ptid));
+        coltok[ptid] = t0;
+      }
+      if (ptid + 96 < KC) {
+        t1 = tok_of(actual_slot(p, cstart + j * KC + ptid + 96));
         coltok[ptid + 96] = t1;
       }
       if (group_sync_stop()) { live = false; break; }
       if (ptid == 0) mbar_arrive(bar(C::kBarTokFull + s));
-      const uint32_t c1 = sbase + C::kOffC + s * 2 * C::kTileBytes, c2 = c1 + C::kTileBytes;
+      const uint32_t c1 = sbase + C::kOffC + s * 2 * C::kColBytes, c2 = c1 + C::kColBytes;
       if (kKeys) {
         // per-query vectors of this head travel with the tile
         const float* lse_h = p.lse + ((size_t)b * p.Hq + hq) * p.n;
         const float* del_h = p.delta + ((size_t)b * p.Hq + hq) * p.n;
-        asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(colvec + 4 * ptid), "l"(lse_h + t0) : "memory");
-        asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(colvec + 4 * (kTile + ptid)), "l"(del_h + t0) : "memory");
-        if (ptid < 32) {
+        if (ptid < KC) {
+          asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(colvec + 4 * ptid), "l"(lse_h + t0) : "memory");
+          asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(colvec + 4 * (kTile + ptid)), "l"(del_h + t0) : "memory");
+        }
+        if (ptid + 96 < KC) {
           asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(colvec + 4 * (ptid + 96)), "l"(lse_h + t1) : "memory");
           asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(colvec + 4 * (kTile + ptid + 96)), "l"(del_h + t1) : "memory");
         }
-        gather(qg + b * p.qs[0] + hq * p.qs[1], p.qs[2], coltok, c1);
-        gather(dyg + b * p.qs[0] + hq * p.qs[1], p.qs[2], coltok, c2);
+        gather(qg + b * p.qs[0] + hq * p.qs[1], p.qs[2], coltok, c1, KC);
+        gather(dyg + b * p.qs[0] + hq * p.qs[1], p.qs[2], coltok, c2, KC);
       } else {
-        gather(kg + b * p.ks[0] + hk * p.ks[1], p.ks[2], coltok, c1);
-        gather(vg + b * p.ks[0] + hk * p.ks[1], p.ks[2], coltok, c2);
+        gather(kg + b * p.ks[0] + hk * p.ks[1], p.ks[2], coltok, c1, KC);
+        gather(vg + b * p.ks[0] + hk * p.ks[1], p.ks[2], coltok, c2, KC);
       }
       signal(bar(C::kBarCFull + s));
     }
@@ -236,30 +251,31 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_tc_kernel(const __grid_con
   } else if (warp == 0) {
     // -------------------------------------------------------------- MMA issuer (warp 0)
     if (lane == 0) {
-      constexpr uint32_t idesc_s = instr_desc(kTile, kTile, false);
+      constexpr uint32_t idesc_s = instr_desc(kTile, KC, false);
       constexpr uint32_t idesc_acc = instr_desc(kTile, D, true);
       constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
       constexpr uint32_t kLoK = (16u >> 4) << 16;                        // K-major operands
-      constexpr uint32_t kLoMN = ((uint32_t)C::kChunkBytes >> 4) << 16;  // column tile as [k][n]
-      constexpr uint32_t kBlock = C::kChunkBytes >> 4;   // next 64 columns of a K-major tile
+      constexpr uint32_t kLoMN = ((uint32_t)C::kColChunkBytes >> 4) << 16;  // column tile as [k][n]
+      constexpr uint32_t kBlockR = C::kChunkBytes >> 4;     // next 64 columns of a row tile
+      constexpr uint32_t kBlockC = C::kColChunkBytes >> 4;  // next 64 columns of a column tile
       const uint64_t r1 = desc64(((sbase + C::kOffR) >> 4) | kLoK, kDescHi);
       const uint64_t r2 = desc64(((sbase + C::kOffR + C::kTileBytes) >> 4) | kLoK, kDescHi);
       // X (128 x 128, fp32, tensor memory column col) = A B^T, both tiles K-major, K = D
       auto product = [&](uint32_t col, uint64_t a, uint32_t b_addr) {
         const uint64_t bd = desc64((b_addr >> 4) | kLoK, kDescHi);
         mma_ss_x4(tmem + col, a, bd, idesc_s, 0u);
-        if (D == 128) mma_ss_x4(tmem + col, a + kBlock, bd + kBlock, idesc_s, 1u);
+        if (D == 128) mma_ss_x4(tmem + col, a + kBlockR, bd + kBlockC, idesc_s, 1u);
       };
       // acc (128 x D, tensor memory column col) += X (bf16 pairs at column xcol) * tile
       auto accumulate = [&](uint32_t col, uint32_t xcol, uint32_t b_addr, uint32_t acc0) {
         const uint64_t bd = desc64((b_addr >> 4) | kLoMN, kDescHi);
         mma_ts_x4(tmem + col, tmem + xcol, bd, idesc_acc, acc0);
-        mma_ts_x4(tmem + col, tmem + xcol + 32, bd + 512, idesc_acc, 1u);
+        if (KC == 128) mma_ts_x4(tmem + col, tmem + xcol + 32, bd + 512, idesc_acc, 1u);
       };
       bool ok = mbar_wait(bar(C::kBarRFull), 0, gave_up, p.status);
       for (int it = 0; it < iters && ok; ++it) {
         const int s = it & 1;
-        const uint32_t c1 = sbase + C::kOffC + s * 2 * C::kTileBytes, c2 = c1 + C::kTileBytes;
+        const uint32_t c1 = sbase + C::kOffC + s * 2 * C::kColBytes, c2 = c1 + C::kColBytes;
         ok = mbar_wait(bar(C::kBarCFull + s), (it >> 1) & 1u, gave_up, p.status);
         if (!ok) break;
         fence_proxy_async();
@@ -309,7 +325,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_tc_kernel(const __grid_con
       if (!ok) break;
       tc_fence_after();
       // visible columns of this row: one interval [lo, lo + span], cut by the token order
-      const int cb = cstart + j * kTile;
+      const int cb = cstart + j * KC;
       int lo, hi;
       if (p.one_sided) {
         if (kKeys) { lo = rslot - cb; hi = p.full_range ? p.n - 1 - cb : rslot + (p.w - 1) - cb; }
@@ -325,7 +341,7 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_tc_kernel(const __grid_con
       const int32_t* coltok = reinterpret_cast<const int32_t*>(smem + C::kOffColTok) + s * kTile;
       const float* colvec = reinterpret_cast<const float*>(smem + C::kOffColVec) + s * 2 * kTile;
 #pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 0; c < KC / 32; ++c) {
         uint32_t sv[32], dv[32];
         tmem_ld32(trow + C::kColS + 32 * c, sv);
         tmem_ld32(trow + C::kColP + 32 * c, dv);
@@ -430,18 +446,30 @@ __global__ void __launch_bounds__(kBwdThreads, 1) bwd_tc_kernel(const __grid_con
 
 // ---------------------------------------------------------------------------- host
 
-template <int D>
+template <int D, int KC>
 cudaError_t launch_branch(const BwdTcParams& p, cudaStream_t st) {
-  const int smem = BCfg<D>::kBytes;
-  cudaError_t e = cudaFuncSetAttribute(bwd_tc_kernel<D, 0>,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  const int smem0 = BCfg<D, KC, 0>::kBytes, smem1 = BCfg<D, KC, 1>::kBytes;
+  cudaError_t e = cudaFuncSetAttribute(bwd_tc_kernel<D, KC, 0>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, smem0);
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(bwd_tc_kernel<D, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+  e = cudaFuncSetAttribute(bwd_tc_kernel<D, KC, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           smem1);
   if (e != cudaSuccess) return e;
-  bwd_tc_kernel<D, 0><<<(unsigned)(p.B * p.Hq * p.n_tiles), kBwdThreads, smem, st>>>(p);
-  bwd_tc_kernel<D, 1><<<(unsigned)(p.B * p.Hkv * p.n_tiles), kBwdThreads, smem, st>>>(p);
+  bwd_tc_kernel<D, KC, 0><<<(unsigned)(p.B * p.Hq * p.n_tiles), kBwdThreads, smem0, st>>>(p);
+  bwd_tc_kernel<D, KC, 1><<<(unsigned)(p.B * p.Hkv * p.n_tiles), kBwdThreads, smem1, st>>>(p);
   bump_launches(2);
   return cudaGetLastError();
+}
+
+// Column-tile width: 64 for narrow windows (less band-edge waste, two CTAs per SM at d = 64),
+// else 128.  SA_KEY_BLOCK=64|128 overrides it so tests can run both.
+bool narrow_columns(int w) {
+  static int forced = -1;
+  if (forced < 0) {
+    const char* e = getenv("SA_KEY_BLOCK");
+    forced = !e ? 0 : (e[0] == '6' ? 64 : 128);
+  }
+  return forced ? forced == 64 : w <= 128;
 }
 
 bool bwd_tc_disabled() {
@@ -482,7 +510,10 @@ cudaError_t launch_bwd_tc(const BwdArgs& a, cudaStream_t st) {
     p.scale = a.scale;
     p.scale2 = a.scale * kLog2e;
     for (int i = 0; i < 3; ++i) { p.qs[i] = a.qs[i]; p.ks[i] = a.ks[i]; }
-    const cudaError_t e = a.d == 128 ? launch_branch<128>(p, st) : launch_branch<64>(p, st);
+    const bool narrow = narrow_columns(a.w);
+    const cudaError_t e =
+        a.d == 128 ? (narrow ? launch_branch<128, 64>(p, st) : launch_branch<128, 128>(p, st))
+                   : (narrow ? launch_branch<64, 64>(p, st) : launch_branch<64, 128>(p, st));
     if (e != cudaSuccess) return e;
   }
   return cudaSuccess;

@@ -120,7 +120,8 @@ def test_both_score_block_widths(block):
     import os, subprocess, sys
     env = dict(os.environ, SA_KEY_BLOCK=block)
     r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-m", "gpu", __file__, "-k",
-                        "test_sa_forward_small or test_swa_forward_small or test_gated_forward_small"],
+                        "test_sa_forward_small or test_swa_forward_small or test_gated_forward_small or "
+                        "test_backward_small"],
                        env=env, capture_output=True, text=True)
     assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
 
