@@ -22,8 +22,13 @@
 // windows and, where scores and accumulators then fit in 256 tensor-memory columns, lets two
 // CTAs share an SM so that one CTA's loads and epilogue hide behind the other's products.
 //
-// Warp roles (256 threads): warp 0 MMA issuer and TMEM allocator, warps 1-3 gather
-// producers, warps 4-7 one thread per row.  Every mbarrier wait is bounded.
+// With NBUF = 2 (64-wide column tiles only) the scores of two consecutive column tiles live
+// side by side in tensor memory: the products of tile i+1 run while the row threads work on
+// tile i, and two warpgroups of row threads split a tile's 64 columns.
+//
+// Warp roles: warp 0 MMA issuer and TMEM allocator, warps 1-3 gather producers, then one
+// (NBUF = 1) or two (NBUF = 2) warpgroups with one thread per row.  Every mbarrier wait is
+// bounded.
 #include "sa_bwd_tc.cuh"
 #include "sa_tc_common.cuh"
 
@@ -31,7 +36,6 @@ namespace sa {
 namespace {
 
 constexpr int kTile = 128;
-constexpr int kBwdThreads = 256;
 constexpr int kProducers = 96;
 
 struct BwdTcParams {
@@ -73,13 +77,16 @@ __device__ __forceinline__ int actual_slot(const BwdTcParams& p, int v) {
   return v < 0 ? v + p.n : v;
 }
 
-template <int D, int KC, int MODE>
+template <int D, int KC, int MODE, int NBUF>
 struct BCfg {
+  static_assert(NBUF == 1 || KC == 64, "two score buffers need 64-wide column tiles");
+  static constexpr int kRowWgs = NBUF;                          // warpgroups of row threads
+  static constexpr int kThreads = 128 + 128 * kRowWgs;
   static constexpr int kTileBytes = kTile * D * 2;              // a row-operand tile
   static constexpr int kChunkBytes = kTile * 128;               // its 64-column blocks
   static constexpr int kColBytes = KC * D * 2;                  // a column tile
   static constexpr int kColChunkBytes = KC * 128;
-  static constexpr int kStages = 2;
+  static constexpr int kStages = NBUF == 2 ? 4 : 2;
   static constexpr int kOffR = 0;                               // two row-operand tiles
   static constexpr int kOffC = 2 * kTileBytes;                  // kStages x two column tiles
   static constexpr int kOffRowTok = kOffC + kStages * 2 * kColBytes;
@@ -88,24 +95,25 @@ struct BCfg {
   static constexpr int kOffBar = kOffColVec + kStages * 2 * kTile * 4;
   static constexpr int kBarRFull = 0, kBarCFull = 1, kBarCEmpty = kBarCFull + kStages,
                        kBarTokFull = kBarCEmpty + kStages, kBarSFull = kBarTokFull + kStages,
-                       kBarPReady = kBarSFull + 1, kBarODone = kBarPReady + 1,
+                       kBarPReady = kBarSFull + NBUF, kBarODone = kBarPReady + NBUF,
                        kNumBars = kBarODone + 1;
   static constexpr int kOffMisc = kOffBar + kNumBars * 8;
   static constexpr int kBytes = kOffMisc + 16;
-  // tensor memory columns: S and dS at 0, dP and P at KC, accumulators from 2 KC
-  static constexpr uint32_t kColS = 0, kColP = KC, kColAcc = 2 * KC;
-  static constexpr uint32_t kColsUsed = 2 * KC + (MODE == 1 ? 2 : 1) * D;
+  // tensor memory columns: S and dS (NBUF buffers of KC) at 0, then dP and P, then the
+  // accumulators
+  static constexpr uint32_t kColS = 0, kColP = KC * NBUF, kColAcc = 2 * KC * NBUF;
+  static constexpr uint32_t kColsUsed = 2 * KC * NBUF + (MODE == 1 ? 2 : 1) * D;
   static constexpr uint32_t kTmemCols = kColsUsed <= 256 ? 256 : 512;
   static constexpr int kCtasPerSm = (kTmemCols == 256 && kBytes <= 110 * 1024) ? 2 : 1;
   static_assert(kBytes <= 232448, "shared memory");
 };
 
 // MODE 0: rows are queries (dQ).  MODE 1: rows are keys (dK, dV).
-template <int D, int KC, int MODE>
-__global__ void __launch_bounds__(kBwdThreads, BCfg<D, KC, MODE>::kCtasPerSm)
+template <int D, int KC, int MODE, int NBUF>
+__global__ void __launch_bounds__(BCfg<D, KC, MODE, NBUF>::kThreads, BCfg<D, KC, MODE, NBUF>::kCtasPerSm)
 bwd_tc_kernel(const __grid_constant__ BwdTcParams p) {
   extern __shared__ __align__(1024) uint8_t smem[];
-  using C = BCfg<D, KC, MODE>;
+  using C = BCfg<D, KC, MODE, NBUF>;
   constexpr uint32_t kTmemCols = C::kTmemCols;
   constexpr bool kKeys = MODE == 1;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -136,7 +144,7 @@ bwd_tc_kernel(const __grid_constant__ BwdTcParams p) {
   if (threadIdx.x == 0) {
     *gave_up = 0;
     for (int i = 0; i < C::kNumBars; ++i)
-      mbar_init(bar(i), i == C::kBarPReady ? kTile
+      mbar_init(bar(i), (i >= C::kBarPReady && i < C::kBarODone) ? kTile * C::kRowWgs
                         : (i == C::kBarRFull || (i >= C::kBarCFull && i < C::kBarCEmpty))
                             ? kProducers : 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -208,11 +216,11 @@ bwd_tc_kernel(const __grid_constant__ BwdTcParams p) {
       signal(bar(C::kBarRFull));
     }
     for (int it = 0; it < iters && live; ++it) {
-      const int s = it & 1;
+      const int s = it % C::kStages;
       const int j = kKeys ? it % T : it, gi = kKeys ? it / T : 0;
       const int hq = kKeys ? hk * p.G + gi : hr;
       if (it >= C::kStages)
-        mbar_wait(bar(C::kBarCEmpty + s), ((it >> 1) - 1) & 1u, gave_up, p.status);
+        mbar_wait(bar(C::kBarCEmpty + s), (it / C::kStages - 1) & 1u, gave_up, p.status);
       int32_t* coltok = reinterpret_cast<int32_t*>(smem + C::kOffColTok) + s * kTile;
       const uint32_t colvec = sbase + C::kOffColVec + s * 2 * kTile * 4;
       int t0 = 0, t1 = 0;
@@ -272,25 +280,38 @@ bwd_tc_kernel(const __grid_constant__ BwdTcParams p) {
         mma_ts_x4(tmem + col, tmem + xcol, bd, idesc_acc, acc0);
         if (KC == 128) mma_ts_x4(tmem + col, tmem + xcol + 32, bd + 512, idesc_acc, 1u);
       };
-      bool ok = mbar_wait(bar(C::kBarRFull), 0, gave_up, p.status);
-      for (int it = 0; it < iters && ok; ++it) {
-        const int s = it & 1;
+      // scores of column tile `it` into buffer it % NBUF
+      auto scores = [&](int it) {
+        const int s = it % C::kStages;
         const uint32_t c1 = sbase + C::kOffC + s * 2 * C::kColBytes, c2 = c1 + C::kColBytes;
-        ok = mbar_wait(bar(C::kBarCFull + s), (it >> 1) & 1u, gave_up, p.status);
-        if (!ok) break;
+        if (!mbar_wait(bar(C::kBarCFull + s), (it / C::kStages) & 1u, gave_up, p.status))
+          return false;
         fence_proxy_async();
         tc_fence_after();
-        product(C::kColS, r1, c1);
-        product(C::kColP, r2, c2);
-        tc_commit(bar(C::kBarSFull));
-        ok = mbar_wait(bar(C::kBarPReady), it & 1u, gave_up, p.status);
+        const uint32_t buf = (it % NBUF) * KC;
+        product(C::kColS + buf, r1, c1);
+        product(C::kColP + buf, r2, c2);
+        tc_commit(bar(C::kBarSFull + it % NBUF));
+        return true;
+      };
+      bool ok = mbar_wait(bar(C::kBarRFull), 0, gave_up, p.status);
+      if (ok && NBUF == 2) ok = scores(0);
+      for (int it = 0; it < iters && ok; ++it) {
+        const int s = it % C::kStages;
+        const uint32_t c1 = sbase + C::kOffC + s * 2 * C::kColBytes, c2 = c1 + C::kColBytes;
+        // NBUF = 2: the next tile's scores go ahead of this tile's accumulation
+        if (NBUF == 2) { if (it + 1 < iters) ok = scores(it + 1); }
+        else ok = scores(it);
+        if (!ok) break;
+        ok = mbar_wait(bar(C::kBarPReady + it % NBUF), (it / NBUF) & 1u, gave_up, p.status);
         if (!ok) break;
         tc_fence_after();
+        const uint32_t buf = (it % NBUF) * KC;
         if (kKeys) {
-          accumulate(C::kColAcc, C::kColP, c2, it > 0);        // dV += (g P)^T dY
-          accumulate(C::kColAcc + D, C::kColS, c1, it > 0);    // dK += dS^T Q
+          accumulate(C::kColAcc, C::kColP + buf, c2, it > 0);        // dV += (g P)^T dY
+          accumulate(C::kColAcc + D, C::kColS + buf, c1, it > 0);    // dK += dS^T Q
         } else {
-          accumulate(C::kColAcc, C::kColS, c1, it > 0);        // dQ += dS K
+          accumulate(C::kColAcc, C::kColS + buf, c1, it > 0);        // dQ += dS K
         }
         tc_commit(bar(C::kBarCEmpty + s));
       }
@@ -298,8 +319,9 @@ bwd_tc_kernel(const __grid_constant__ BwdTcParams p) {
     }
     __syncwarp();
   } else {
-    // ------------------------------------------------- one thread per row (warps 4-7)
-    const int row = threadIdx.x - 128;                  // 0..127 == TMEM lane
+    // ------------------------------------------------- row threads (from warp 4 on)
+    const int wg = (warp - 4) >> 2;                     // which warpgroup of row threads
+    const int row = (threadIdx.x - 128) & 127;          // 0..127 == TMEM lane
     const uint32_t trow = tmem + ((uint32_t)(row & ~31) << 16);
     const int rslot = r0 + row;
     const bool row_valid = rslot < p.n;
@@ -314,16 +336,32 @@ bwd_tc_kernel(const __grid_constant__ BwdTcParams p) {
       delta_r = p.delta[o];
       if (p.gate_logit) g = 1.f / (1.f + __expf(-p.gate_logit[hr]));
     }
+    // Two warpgroups share a tile: the bf16 results of one overwrite score columns the other
+    // reads, so every row thread loads before any stores.  The barrier also agrees on whether
+    // to stop, so that all of them leave the loop together.
+    auto rows_sync_stop = [&](bool stop) {
+      uint32_t any;
+      asm volatile(
+          "{\n\t.reg .pred p, q;\n\t"
+          "setp.ne.u32 q, %1, 0;\n\t"
+          "bar.red.or.pred p, 2, 256, q;\n\t"
+          "selp.u32 %0, 1, 0, p;\n\t}"
+          : "=r"(any)
+          : "r"((uint32_t)stop)
+          : "memory");
+      return any != 0;
+    };
     bool ok = true;
     for (int it = 0; it < iters; ++it) {
-      const int s = it & 1;
+      const int s = it % C::kStages;
+      const uint32_t buf = (it % NBUF) * KC;
       const int j = kKeys ? it % T : it;
       if (kKeys && p.gate_logit) g = 1.f / (1.f + __expf(-p.gate_logit[hk * p.G + it / T]));
-      ok = mbar_wait(bar(C::kBarTokFull + s), (it >> 1) & 1u, gave_up, p.status);
-      if (ok) ok = mbar_wait(bar(C::kBarSFull), it & 1u, gave_up, p.status);
+      ok = mbar_wait(bar(C::kBarTokFull + s), (it / C::kStages) & 1u, gave_up, p.status);
+      if (ok) ok = mbar_wait(bar(C::kBarSFull + it % NBUF), (it / NBUF) & 1u, gave_up, p.status);
       ok = __all_sync(0xffffffffu, ok);   // the tensor-memory accesses below are warp-collective
-      if (!ok) break;
-      tc_fence_after();
+      if (C::kRowWgs == 1 && !ok) break;
+      if (ok) tc_fence_after();
       // visible columns of this row: one interval [lo, lo + span], cut by the token order
       const int cb = cstart + j * KC;
       int lo, hi;
@@ -341,11 +379,14 @@ bwd_tc_kernel(const __grid_constant__ BwdTcParams p) {
       const int32_t* coltok = reinterpret_cast<const int32_t*>(smem + C::kOffColTok) + s * kTile;
       const float* colvec = reinterpret_cast<const float*>(smem + C::kOffColVec) + s * 2 * kTile;
 #pragma unroll 1
-      for (int c = 0; c < KC / 32; ++c) {
+      for (int c = wg; c < KC / 32; c += C::kRowWgs) {
         uint32_t sv[32], dv[32];
-        tmem_ld32(trow + C::kColS + 32 * c, sv);
-        tmem_ld32(trow + C::kColP + 32 * c, dv);
-        tmem_wait_ld();
+        if (ok) {
+          tmem_ld32(trow + C::kColS + buf + 32 * c, sv);
+          tmem_ld32(trow + C::kColP + buf + 32 * c, dv);
+          tmem_wait_ld();
+        }
+        if (C::kRowWgs == 2 && rows_sync_stop(!ok)) { ok = false; break; }
         uint32_t ds_pk[16], p_pk[16];
 #pragma unroll
         for (int x = 0; x < 32; x += 4) {
@@ -382,52 +423,52 @@ bwd_tc_kernel(const __grid_constant__ BwdTcParams p) {
           }
         }
         // bf16 results go back over the columns already consumed (16 c .. 16 c + 15)
-        tmem_st16(trow + C::kColS + 16 * c, ds_pk);
-        if (kKeys) tmem_st16(trow + C::kColP + 16 * c, p_pk);
+        tmem_st16(trow + C::kColS + buf + 16 * c, ds_pk);
+        if (kKeys) tmem_st16(trow + C::kColP + buf + 16 * c, p_pk);
       }
+      if (!ok) break;
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(bar(C::kBarPReady));
+      mbar_arrive(bar(C::kBarPReady + it % NBUF));
     }
 
     if (ok) ok = mbar_wait(bar(C::kBarODone), 0, gave_up, p.status);
     ok = __all_sync(0xffffffffu, ok);
     if (ok) {
       tc_fence_after();
-      constexpr int kOuts = kKeys ? 2 : 1;
-#pragma unroll
-      for (int o = 0; o < kOuts; ++o) {
-        // rows = keys: accumulator 0 is dV, 1 is dK
+      // 32-column pieces of the accumulators (rows = keys: dV first, then dK), dealt to the
+      // warpgroups in turn
+      constexpr int kPieces = (kKeys ? 2 : 1) * (D / 32);
+#pragma unroll 1
+      for (int piece = wg; piece < kPieces; piece += C::kRowWgs) {
+        const int o = piece / (D / 32), c = piece % (D / 32);
         __nv_bfloat16* out = (__nv_bfloat16*)(kKeys ? (o == 0 ? p.dv : p.dk) : p.dq);
         const int64_t* st = kKeys ? p.ks : p.qs;
         const int64_t off = b * st[0] + hr * st[1] + (int64_t)rtok * st[2];
+        uint32_t raw[32];
+        tmem_ld32(trow + C::kColAcc + o * D + 32 * c, raw);   // warp-collective
+        tmem_wait_ld();
+        if (row_valid) {
 #pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-          uint32_t raw[32];
-          tmem_ld32(trow + C::kColAcc + o * D + 32 * c, raw);   // warp-collective
-          tmem_wait_ld();
-          if (row_valid) {
+          for (int x8 = 0; x8 < 4; ++x8) {
+            float v8[8];
 #pragma unroll
-            for (int x8 = 0; x8 < 4; ++x8) {
-              float v8[8];
+            for (int x = 0; x < 8; ++x) v8[x] = __uint_as_float(raw[8 * x8 + x]);
+            uint4* dst = reinterpret_cast<uint4*>(out + off + 32 * c + 8 * x8);
+            if (p.accumulate) {
+              const uint4 old = *dst;
+              const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&old);
 #pragma unroll
-              for (int x = 0; x < 8; ++x) v8[x] = __uint_as_float(raw[8 * x8 + x]);
-              uint4* dst = reinterpret_cast<uint4*>(out + off + 32 * c + 8 * x8);
-              if (p.accumulate) {
-                const uint4 old = *dst;
-                const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&old);
-#pragma unroll
-                for (int x = 0; x < 4; ++x) {
-                  v8[2 * x] += __low2float(h2[x]);
-                  v8[2 * x + 1] += __high2float(h2[x]);
-                }
+              for (int x = 0; x < 4; ++x) {
+                v8[2 * x] += __low2float(h2[x]);
+                v8[2 * x + 1] += __high2float(h2[x]);
               }
-              uint4 pk;
-              __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&pk);
-#pragma unroll
-              for (int x = 0; x < 4; ++x) h2[x] = __floats2bfloat162_rn(v8[2 * x], v8[2 * x + 1]);
-              *dst = pk;
             }
+            uint4 pk;
+            __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&pk);
+#pragma unroll
+            for (int x = 0; x < 4; ++x) h2[x] = __floats2bfloat162_rn(v8[2 * x], v8[2 * x + 1]);
+            *dst = pk;
           }
         }
       }
@@ -446,30 +487,34 @@ bwd_tc_kernel(const __grid_constant__ BwdTcParams p) {
 
 // ---------------------------------------------------------------------------- host
 
-template <int D, int KC>
+template <int D, int KC, int NBUF>
 cudaError_t launch_branch(const BwdTcParams& p, cudaStream_t st) {
-  const int smem0 = BCfg<D, KC, 0>::kBytes, smem1 = BCfg<D, KC, 1>::kBytes;
-  cudaError_t e = cudaFuncSetAttribute(bwd_tc_kernel<D, KC, 0>,
-                                       cudaFuncAttributeMaxDynamicSharedMemorySize, smem0);
+  using C0 = BCfg<D, KC, 0, NBUF>;
+  using C1 = BCfg<D, KC, 1, NBUF>;
+  cudaError_t e = cudaFuncSetAttribute(bwd_tc_kernel<D, KC, 0, NBUF>,
+                                       cudaFuncAttributeMaxDynamicSharedMemorySize, C0::kBytes);
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(bwd_tc_kernel<D, KC, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           smem1);
+  e = cudaFuncSetAttribute(bwd_tc_kernel<D, KC, 1, NBUF>,
+                           cudaFuncAttributeMaxDynamicSharedMemorySize, C1::kBytes);
   if (e != cudaSuccess) return e;
-  bwd_tc_kernel<D, KC, 0><<<(unsigned)(p.B * p.Hq * p.n_tiles), kBwdThreads, smem0, st>>>(p);
-  bwd_tc_kernel<D, KC, 1><<<(unsigned)(p.B * p.Hkv * p.n_tiles), kBwdThreads, smem1, st>>>(p);
+  bwd_tc_kernel<D, KC, 0, NBUF><<<(unsigned)(p.B * p.Hq * p.n_tiles), C0::kThreads, C0::kBytes, st>>>(p);
+  bwd_tc_kernel<D, KC, 1, NBUF><<<(unsigned)(p.B * p.Hkv * p.n_tiles), C1::kThreads, C1::kBytes, st>>>(p);
   bump_launches(2);
   return cudaGetLastError();
 }
 
-// Column-tile width: 64 for narrow windows (less band-edge waste, two CTAs per SM at d = 64),
-// else 128.  SA_KEY_BLOCK=64|128 overrides it so tests can run both.
-bool narrow_columns(int w) {
+// Kernel shape: 0 = 64-wide column tiles, one score buffer (narrow windows: least band-edge
+// waste, two CTAs per SM at d = 64); 1 = 64-wide tiles, two score buffers and two row
+// warpgroups (products of the next tile overlap the row work of this one); 2 = 128-wide
+// tiles, one buffer.  SA_KEY_BLOCK=64|128 forces shape 0 or 2 so tests can run every shape.
+int bwd_shape(int w) {
   static int forced = -1;
   if (forced < 0) {
     const char* e = getenv("SA_KEY_BLOCK");
     forced = !e ? 0 : (e[0] == '6' ? 64 : 128);
   }
-  return forced ? forced == 64 : w <= 128;
+  if (forced) return forced == 64 ? 0 : 2;
+  return w <= 128 ? 0 : 1;
 }
 
 bool bwd_tc_disabled() {
@@ -510,10 +555,14 @@ cudaError_t launch_bwd_tc(const BwdArgs& a, cudaStream_t st) {
     p.scale = a.scale;
     p.scale2 = a.scale * kLog2e;
     for (int i = 0; i < 3; ++i) { p.qs[i] = a.qs[i]; p.ks[i] = a.ks[i]; }
-    const bool narrow = narrow_columns(a.w);
-    const cudaError_t e =
-        a.d == 128 ? (narrow ? launch_branch<128, 64>(p, st) : launch_branch<128, 128>(p, st))
-                   : (narrow ? launch_branch<64, 64>(p, st) : launch_branch<64, 128>(p, st));
+    const int shape = bwd_shape(a.w);
+    cudaError_t e;
+    if (a.d == 128)
+      e = shape == 0 ? launch_branch<128, 64, 1>(p, st)
+          : shape == 1 ? launch_branch<128, 64, 2>(p, st) : launch_branch<128, 128, 1>(p, st);
+    else
+      e = shape == 0 ? launch_branch<64, 64, 1>(p, st)
+          : shape == 1 ? launch_branch<64, 64, 2>(p, st) : launch_branch<64, 128, 1>(p, st);
     if (e != cudaSuccess) return e;
   }
   return cudaSuccess;
