@@ -369,6 +369,31 @@ def extras(args, c, wl, sa, torch, dev, host, perm, inv, ws, y, pk):
     del t5, saved, bout, bws
     torch.cuda.empty_cache()
 
+    # the shape of the paper's efficiency table (Sec. 4.3, Table 3: B=16, H=16, d_h=64, w=256,
+    # forward + backward of single-path SA); the paper's A100 / FlexAttention times are context
+    t3 = {}
+    paper_ms = {2048: 5.4, 4096: 7.9, 8192: 15.2, 16384: 29.6, 32768: 52.8}
+    for n3 in (2048, 8192, 32768):
+        c3 = wl.Workload("table3", "bf16", 16, 16, 16, n3, 64, 256, seed=9, ops="gated_fwd_bwd")
+        d3 = {k_: v_.cuda() for k_, v_ in wl.draw(c3).items()}
+        p3, i3 = sa.sa_make_perm(9, 0, c3.B, c3.n)
+        y3 = torch.empty_like(d3["q"])
+        l3 = torch.empty(c3.B, c3.Hq, c3.n, dtype=torch.float32, device="cuda")
+        w3 = torch.empty(sa.sa_workspace_bytes(sa.make_problem(d3["q"], d3["k"], c3.w, c3.flags),
+                                               sa.OP_BACKWARD), dtype=torch.uint8, device="cuda")
+        o3 = {}
+
+        def fb3():
+            sa.sa_forward(d3["q"], d3["k"], d3["v"], p3, i3, c3.w, c3.flags, y=y3, lse=l3)
+            r = sa.sa_backward(d3["q"], d3["k"], d3["v"], p3, i3, None, y3, None, l3, None,
+                               d3["dy"], c3.w, c3.flags, ws=w3, out=o3)
+            o3.update(zip(("dq", "dk", "dv", "dgate"), r))
+        t3[str(n3)] = {"sa_fwd_bwd_ms": event_ms(fb3, 3, 2, torch),
+                       "paper_a100_flexattention_ms": paper_ms[n3]}
+        del d3, y3, l3, w3, o3
+        torch.cuda.empty_cache()
+    res["table3_shape_B16_H16_d64_w256"] = t3
+
     rate, dt, rows, threads = oracle_sample_rate(c, host, 196608)
     res["cpu_baseline"] = {
         "value": rate, "unit": "tokens/s", "cores": threads, "kind": "oracle",

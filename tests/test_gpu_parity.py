@@ -363,6 +363,33 @@ def test_coverage_bit_exact(n, w, flags, L):
         assert np.array_equal(reach.cpu().numpy(), oreach)
 
 
+def test_coverage_study_sa_against_swa_and_prop2_bound():
+    # Fig. 2 (left) setting: n = 2048, w = 32.  Seed-averaged reach of SA per layer against the
+    # expansion bound of Prop. 2, and against plain SWA, whose reach grows by 2h per layer.
+    n, w, L, seeds, src = 2048, 32, 6, 24, 5
+    h = (w + 1) // 2 - 1
+    band = 2 * h + 1
+    pr = (band - 1) / (n - 1)
+    sizes = np.zeros((seeds, L))
+    for s_ in range(seeds):
+        pl = [sa.sa_make_perm(7000 + s_, l, 1, n) for l in range(L)]
+        perm = torch.cat([a_ for a_, _ in pl]).contiguous()
+        inv = torch.cat([b_ for _, b_ in pl]).contiguous()
+        nnz, rc, reach = sa.sa_coverage(perm, inv, w, 0, src)
+        sizes[s_] = reach.cpu().numpy()
+        assert int(rc.min()) == band and int(rc.max()) == band
+    assert np.all(sizes[:, 0] == band) and np.all(np.diff(sizes, axis=1) >= 0)
+    mean = sizes.mean(axis=0)
+    for l in range(L - 1):
+        r = sizes[:, l]
+        assert mean[l + 1] >= 0.97 * (r + (n - r) * (1 - (1 - pr) ** r)).mean()
+    assert mean[3] > 0.99 * n                       # full coverage in O(log_w n) layers
+    ident = torch.arange(n, dtype=torch.int32, device="cuda").repeat(L, 1).contiguous()
+    _, _, swa_reach = sa.sa_coverage(ident, ident, w, 0, src)
+    assert swa_reach.cpu().tolist() == [min(n, 2 * (l + 1) * h + 1) for l in range(L)]
+    assert mean[2] > 10 * swa_reach[2].item()       # SA has spread far beyond the local window
+
+
 # ----------------------------------------------------------------------- status
 
 def test_validate_perm_reports_a_non_bijection():
