@@ -499,6 +499,14 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
       const bool row_valid = cur.row_valid;
       const int q_tok = cur.q_tok;
       const int qcmp = (p.causal && !p.one_sided) ? q_tok : 0x7fffffff;
+      if (p.gate_logits && p.y_other && row_valid) {
+        // the epilogue will read the other branch's row: start bringing it into L2 now
+        const __nv_bfloat16* orow = (const __nv_bfloat16*)p.y_other + b * p.qs[0] +
+                                    cur.hq * p.qs[1] + (int64_t)q_tok * p.qs[2];
+#pragma unroll
+        for (int x = 0; x < D * 2 / 128; ++x)
+          asm volatile("prefetch.global.L2 [%0];" ::"l"(orow + 64 * x));
+      }
       float m = -INFINITY, l = 0.f;
       bool started = false;
 
