@@ -32,12 +32,25 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
 }
 
 // Bounded wait.  Returns false when the limit ran out or another thread already gave up.
+// try_wait that lets the hardware park the thread for up to `ns` nanoseconds while the phase
+// is incomplete, instead of returning at once: a waiting warp then costs next to no issue slots.
+__device__ __forceinline__ bool mbar_try_parked(uint32_t bar, uint32_t parity, uint32_t ns) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity), "r"(ns)
+      : "memory");
+  return ok != 0;
+}
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* gave_up,
                                           int* status) {
   if (mbar_try(bar, parity)) return true;
   const long long t0 = clock64();
   while (true) {
-    if (mbar_try(bar, parity)) return true;
+    if (mbar_try_parked(bar, parity, 2000u)) return true;
     if (*gave_up) return false;
     if (clock64() - t0 > kWaitCycles) {
       *gave_up = 1;
