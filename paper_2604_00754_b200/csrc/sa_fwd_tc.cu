@@ -255,12 +255,36 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
     auto wait_free = [&](uint32_t mb, uint32_t parity) {
       mbar_wait(mb, parity, gave_up, p.status);     // a failure sets *gave_up
     };
+    // The rows of a tile are dealt to the three warps in groups of kRpi (group g to warp
+    // g mod 3).  A warp takes four of its groups per pass (g, g+3, g+6, g+9): over a pass the
+    // swizzle term of each of the four is the same in every pass (g advances by 12, and the
+    // term only depends on g modulo 8 / kRpi), so it is prepared once per thread and the
+    // destination of a copy is one addition away from the pass's base.
+    constexpr int kGroups = kTile / kRpi;
+    uint32_t sw[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int r7 = ((warp - 1 + 3 * k) * kRpi + sub) & 7;
+      sw[k] = (uint32_t)(((chunk & 7) ^ r7) << 4) + (uint32_t)(3 * k * kRpi * 128);
+    }
     auto gather = [&](const __nv_bfloat16* base, int64_t tok_stride, const int32_t* toks,
                       uint32_t dst_tile) {
-#pragma unroll 4
-      for (int grp = warp - 1; grp < kTile / kRpi; grp += 3) {
+      const __nv_bfloat16* src0 = base + chunk * 8;
+      const uint32_t dst0 = dst_tile + dst_lane + sub * 128;
+      int grp = warp - 1;
+      for (; grp + 9 < kGroups; grp += 12) {
+        const int32_t* tk = toks + grp * kRpi + sub;
+        const uint32_t d = dst0 + grp * (kRpi * 128);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const __nv_bfloat16* src = src0 + (int64_t)tk[3 * k * kRpi] * tok_stride;
+          asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d + sw[k]), "l"(src)
+                       : "memory");
+        }
+      }
+      for (; grp < kGroups; grp += 3) {
         const int r = grp * kRpi + sub;
-        const __nv_bfloat16* src = base + (int64_t)toks[r] * tok_stride + chunk * 8;
+        const __nv_bfloat16* src = src0 + (int64_t)toks[r] * tok_stride;
         const uint32_t dst = dst_tile + dst_lane + r * 128 + (((chunk & 7) ^ (r & 7)) << 4);
         asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
       }
