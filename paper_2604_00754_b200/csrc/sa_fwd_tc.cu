@@ -269,7 +269,9 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
     }
     auto gather = [&](const __nv_bfloat16* base, int64_t tok_stride, const int32_t* toks,
                       uint32_t dst_tile) {
-      const __nv_bfloat16* src0 = base + chunk * 8;
+      // token and token stride are both below 2^31: one 32 x 32 -> 64 bit multiply per row
+      const uint32_t ts = (uint32_t)tok_stride * 2u;      // bytes
+      const char* src0 = reinterpret_cast<const char*>(base + chunk * 8);
       const uint32_t dst0 = dst_tile + dst_lane + sub * 128;
       int grp = warp - 1;
       for (; grp + 9 < kGroups; grp += 12) {
@@ -277,14 +279,14 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
         const uint32_t d = dst0 + grp * (kRpi * 128);
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
-          const __nv_bfloat16* src = src0 + (int64_t)tk[3 * k * kRpi] * tok_stride;
+          const char* src = src0 + (uint64_t)(uint32_t)tk[3 * k * kRpi] * ts;
           asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d + sw[k]), "l"(src)
                        : "memory");
         }
       }
       for (; grp < kGroups; grp += 3) {
         const int r = grp * kRpi + sub;
-        const __nv_bfloat16* src = src0 + (int64_t)toks[r] * tok_stride;
+        const char* src = src0 + (uint64_t)(uint32_t)toks[r] * ts;
         const uint32_t dst = dst_tile + dst_lane + r * 128 + (((chunk & 7) ^ (r & 7)) << 4);
         asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
       }
@@ -755,6 +757,7 @@ bool tc_disabled() {
 bool tc_forward_supported(const FwdArgs& a, int dtype) {
   if (tc_disabled() || dtype != SA_BF16 || (a.d != 128 && a.d != 64)) return false;
   if (a.n < 1 || (int64_t)a.B * a.Hq * ((a.n + kTile - 1) / kTile) > 0x3fffffff) return false;
+  if (a.qs[2] >= (1ll << 30) || a.ks[2] >= (1ll << 30)) return false;   // 32-bit row strides
   return true;
 }
 
