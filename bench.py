@@ -273,7 +273,7 @@ def main():
     # is under profiles/), scaled by n because every tensor grows in proportion to it.
     traffic = None
     if (c.B, c.Hq, c.Hkv, c.d, c.w) == (1, 32, 8, 128, 1024):
-        traffic = 194426624.0 * c.n / 8192
+        traffic = 196676352.0 * c.n / 8192
     sustained = args.steps * ms_per_step > 1500.0
     peak = pk["bf16_tflops_sustained"] if sustained else pk["bf16_tflops"]
     line = {
