@@ -322,24 +322,22 @@ def extras(args, c, wl, sa, torch, dev, host, perm, inv, ws, y, pk):
     res["sa_overhead_vs_swa"] = sa_ms / swa_ms - 1.0
     res["make_perm_ms"] = perm_ms
 
-    # end to end: host (pinned) inputs -> device, the step, result back to the host
+    # end to end through the host-memory API: pinned host inputs -> device, fresh permutation,
+    # gated forward, result back to pinned host memory; the KV-head groups are pipelined so
+    # that copies in, kernels and copies out overlap
+    from paper_2604_00754_b200 import host as sa_host
     hy = torch.empty_like(host["q"]).pin_memory()
-    h2d = sum(host[n_].numel() * host[n_].element_size() for n_ in ("q", "k", "v", "gate_logits"))
-    d2h = hy.numel() * hy.element_size()
-    out = {"y": y}
+    hf = sa_host.HostForward(c.B, c.Hq, c.Hkv, c.n, c.d, c.w, c.flags, n_groups=8)
     layer = [1000]
 
     def e2e_step():
-        for n_ in ("q", "k", "v", "gate_logits"):
-            dev[n_].copy_(host[n_], non_blocking=True)
-        sa.sa_make_perm(c.seed, layer[0], c.B, c.n, perm=perm, inv=inv, ws=ws)
-        sa.sa_swa_gated_forward(dev["q"], dev["k"], dev["v"], perm, inv, dev["gate_logits"], c.w,
-                                c.flags, out=out)
-        hy.copy_(y, non_blocking=True)
+        hf.forward(host["q"], host["k"], host["v"], host["gate_logits"], hy, c.seed, layer[0])
         layer[0] += 1
     e2e_ms = event_ms(e2e_step, it, 2, torch)
     res["e2e"] = {"value": c.B * c.n / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms,
-                  "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+                  "h2d_bytes_per_step": hf.h2d_bytes(), "d2h_bytes_per_step": hf.d2h_bytes(),
+                  "api": "host.HostForward.forward, 8 KV-head groups on 3 streams"}
+    del hf
 
     # backward on the pre-training shape (fresh permutation, gated forward saving, backward)
     c5 = wl.C5

@@ -1,0 +1,52 @@
+"""Host-to-host forward: the head grouping (CPU) and, on a GPU, that the pipelined path gives
+the bits of the single device-resident call."""
+import pytest
+import torch
+
+from paper_2604_00754_b200 import host
+
+
+def test_head_groups_cover_every_head_once():
+    for Hq, Hkv, ng in [(32, 8, 8), (32, 8, 3), (12, 12, 5), (4, 1, 8), (16, 4, 1)]:
+        groups = host.head_groups(Hq, Hkv, ng)
+        assert len(groups) <= max(1, min(ng, Hkv))
+        G = Hq // Hkv
+        kv_seen, q_seen = [], []
+        for ka, kb, qa, qb in groups:
+            assert kb > ka and (qa, qb) == (ka * G, kb * G)
+            kv_seen += list(range(ka, kb))
+            q_seen += list(range(qa, qb))
+        assert kv_seen == list(range(Hkv)) and q_seen == list(range(Hq))
+
+
+def test_head_groups_rejects_bad_head_counts():
+    with pytest.raises(ValueError):
+        host.head_groups(10, 4, 2)
+    with pytest.raises(ValueError):
+        host.head_groups(0, 1, 1)
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("n_groups", [1, 3, 4])
+def test_pipelined_forward_equals_single_call(n_groups):
+    from paper_2604_00754_b200 import binding as sa
+    B, Hq, Hkv, n, d, w = 2, 8, 4, 1000, 64, 256
+    g = torch.Generator().manual_seed(11)
+    q = torch.randn(B, Hq, n, d, generator=g).bfloat16().pin_memory()
+    k = torch.randn(B, Hkv, n, d, generator=g).bfloat16().pin_memory()
+    v = torch.randn(B, Hkv, n, d, generator=g).bfloat16().pin_memory()
+    lg = torch.randn(2, Hq, generator=g).pin_memory()
+    hy = torch.empty_like(q).pin_memory()
+    hf = host.HostForward(B, Hq, Hkv, n, d, w, n_groups=n_groups)
+    hf.forward(q, k, v, lg, hy, seed=5, layer=2)
+    torch.cuda.synchronize()
+    perm, inv = sa.sa_make_perm(5, 2, B, n)
+    ref = sa.sa_swa_gated_forward(q.cuda(), k.cuda(), v.cuda(), perm, inv, lg.cuda(), w)
+    assert sa.sa_read_status() == 0
+    assert torch.equal(hy, ref.cpu())
+    # a second call with another layer index draws another permutation
+    hf.forward(q, k, v, lg, hy, seed=5, layer=3)
+    torch.cuda.synchronize()
+    perm, inv = sa.sa_make_perm(5, 3, B, n)
+    ref = sa.sa_swa_gated_forward(q.cuda(), k.cuda(), v.cuda(), perm, inv, lg.cuda(), w)
+    assert torch.equal(hy, ref.cpu())
