@@ -246,3 +246,24 @@ def forward_rows(swa, q, k, v, perm, inv, w, flags, rows, scale=0.0):
         rows.ctypes.data_as(ctypes.c_void_p), y.ctypes.data_as(ctypes.c_void_p),
         lse.ctypes.data_as(ctypes.c_void_p))
     return y, lse
+
+
+def gate_projection(y_sa, w_sa, y_swa=None, w_swa=None):
+    """Projection gates of Eq. 5-6 (App. B, dual-path and single-path attention gate).
+
+    y_*: [rows, dm] attention outputs with the heads concatenated per token; w_*: [dm, dm]
+    weights of a bias-free linear layer (out_features x in_features), so the gate of a path is
+    g = sigmoid(y w^T), per token and per dimension, and the result is
+    g_sa * y_sa (+ g_swa * y_swa for the dual path).  Plain float64 numpy: one matmul, one
+    logistic and one product per path, nothing blocked or fused."""
+    def one(y, w):
+        y = np.asarray(y, dtype=np.float64)
+        w = np.asarray(w, dtype=np.float64)
+        if y.ndim != 2 or w.shape != (y.shape[1], y.shape[1]):
+            raise ValueError("y must be [rows, dm] and w [dm, dm]")
+        g = 1.0 / (1.0 + np.exp(-(y @ w.T)))
+        return g * y
+    out = one(y_sa, w_sa)
+    if y_swa is not None:
+        out = out + one(y_swa, w_swa)
+    return out
