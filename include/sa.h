@@ -174,6 +174,23 @@ sa_status sa_coverage(int32_t L, int32_t n, int32_t w, uint32_t flags, const int
                       const int32_t* inv, int32_t src, int64_t* nnz, int32_t* row_count,
                       int32_t* reach, void* ws, size_t ws_bytes, sa_stream_t stream);
 
+/* Projection gates of Eq. 5-6 (dual path) and of the single-path attention gate of App. B:
+ *   out = sigmoid(y_sa w_sa^T) * y_sa  [+ sigmoid(y_swa w_swa^T) * y_swa],
+ * per token and per dimension, the two sigmoids independent.  y_sa, y_swa, out: device,
+ * [rows, dm] in the run dtype, row r starting ld_y (ld_out) elements after row r-1: the
+ * attention outputs with the heads of a token side by side (sa_forward writes that layout
+ * when given the strides of a [B,n,Hq,d] tensor).  w_sa, w_swa: device, [dm, dm] row-major
+ * (out_features x in_features, a bias-free linear layer), same dtype.  y_swa == NULL selects
+ * the single-path gate (w_swa ignored).  Products accumulate in fp32; the logistic and the
+ * combination are fp32, rounded once to the run dtype.  dtype SA_BF16 with dm a multiple of
+ * 64 and 16-byte aligned rows runs on the tensor cores; every other case on a plain kernel.
+ * Nothing is allocated; inputs are not modified; out may not alias an input.
+ * Errors: SA_ERR_INVALID_ARG (null pointer, rows < 1, dm < 1, ld < dm), SA_ERR_CUDA. */
+sa_status sa_gate_projection_forward(int64_t rows, int32_t dm, int32_t dtype, const void* y_sa,
+                                     const void* y_swa, int64_t ld_y, const void* w_sa,
+                                     const void* w_swa, void* out, int64_t ld_out,
+                                     sa_stream_t stream);
+
 /* Synchronises the stream, returns the device status word (SA_OK, SA_ERR_BAD_PERM or
  * SA_ERR_TIMEOUT) of the current device and clears it. */
 sa_status sa_read_status(sa_stream_t stream);

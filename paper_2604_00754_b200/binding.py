@@ -27,6 +27,7 @@ EXPORTS = [
     "sa_problem_set_contiguous", "sa_workspace_bytes", "sa_make_perm", "sa_forward",
     "sa_swa_forward", "sa_swa_gated_forward", "sa_backward", "sa_coverage", "sa_read_status",
     "sa_status_string", "sa_launch_count", "sa_set_profile_events", "sa_make_perm_static",
+    "sa_gate_projection_forward",
 ]
 
 
@@ -79,6 +80,9 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.sa_swa_gated_forward.argtypes = [pp] + [vp] * 12 + [sz, vp]
     lib.sa_backward.argtypes = [pp] + [vp] * 16 + [sz, vp]
     lib.sa_coverage.argtypes = [i32, i32, i32, u32, vp, vp, i32, vp, vp, vp, vp, sz, vp]
+    lib.sa_gate_projection_forward.argtypes = [ctypes.c_int64, i32, i32, vp, vp, ctypes.c_int64,
+                                               vp, vp, vp, ctypes.c_int64, vp]
+    lib.sa_gate_projection_forward.restype = ctypes.c_int
     lib.sa_read_status.argtypes = [vp]
     for f in ("sa_make_perm", "sa_forward", "sa_swa_forward", "sa_swa_gated_forward",
               "sa_backward", "sa_coverage", "sa_read_status"):
@@ -298,6 +302,37 @@ def sa_coverage(perm, inv, w, flags, src, want_row_count=True, ws=None):
                            _ptr(rc), _ptr(reach), _ptr(ws), ws.numel(), _stream()),
            "sa_coverage")
     return nnz, rc, reach
+
+
+def sa_gate_projection_forward(y_sa, w_sa, y_swa=None, w_swa=None, out=None):
+    """out = sigmoid(y_sa w_sa^T) * y_sa (+ sigmoid(y_swa w_swa^T) * y_swa): Eq. 5-6.
+
+    y_*: [rows, dm] with unit stride along dm (any row pitch, e.g. a [B*n, Hq*d] view of a
+    [B,n,Hq,d] attention output); w_*: contiguous [dm, dm] (out_features x in_features)."""
+    lib = load_library()
+    rows, dm = y_sa.shape
+    if y_sa.dtype == torch.float32:
+        dt = 0
+    elif y_sa.dtype == torch.bfloat16:
+        dt = 1
+    else:
+        raise ValueError("dtype must be float32 or bfloat16")
+    for t in (y_sa, y_swa):
+        if t is not None and (t.dim() != 2 or t.stride(1) != 1 or t.shape != y_sa.shape
+                              or t.stride(0) != y_sa.stride(0) or t.dtype != y_sa.dtype):
+            raise ValueError("y tensors must be [rows, dm] with unit inner stride and one pitch")
+    for t in (w_sa, w_swa):
+        if t is not None and (tuple(t.shape) != (dm, dm) or not t.is_contiguous()
+                              or t.dtype != y_sa.dtype):
+            raise ValueError("w tensors must be contiguous [dm, dm] of the run dtype")
+    if out is None:
+        out = torch.empty(rows, dm, dtype=y_sa.dtype, device=y_sa.device)
+    if out.stride(1) != 1 or tuple(out.shape) != (rows, dm) or out.dtype != y_sa.dtype:
+        raise ValueError("out must be [rows, dm] with unit inner stride")
+    _check(lib.sa_gate_projection_forward(rows, dm, dt, _ptr(y_sa), _ptr(y_swa), y_sa.stride(0),
+                                          _ptr(w_sa), _ptr(w_swa), _ptr(out), out.stride(0),
+                                          _stream()), "sa_gate_projection_forward")
+    return out
 
 
 def sa_read_status() -> int:

@@ -1,0 +1,73 @@
+"""Projection gates of Eq. 5-6 through the C ABI against the float64 oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+
+pytestmark = pytest.mark.gpu
+
+
+def _draw(rows, dm, seed, dtype, pitch=None):
+    g = torch.Generator().manual_seed(seed)
+    pitch = pitch or dm
+    def y():
+        t = torch.randn(rows, pitch, generator=g).to(dtype)
+        return t
+    ws = (dm ** -0.5)
+    return y(), y(), (torch.randn(dm, dm, generator=g) * ws).to(dtype), (torch.randn(dm, dm, generator=g) * ws).to(dtype)
+
+
+def _check(out, ya, wa, yb, wb, dm, tol):
+    want = oracle.gate_projection(ya[:, :dm].double().numpy(), wa.double().numpy(),
+                                  None if yb is None else yb[:, :dm].double().numpy(),
+                                  None if wb is None else wb.double().numpy())
+    got = out.double().cpu().numpy()
+    err = np.abs(got - want)
+    bound = tol * np.maximum(np.abs(want), 1.0)
+    assert (err <= bound).all(), float((err / np.maximum(np.abs(want), 1.0)).max())
+
+
+# bf16 result: one rounding of the output (2^-9 relative) plus fp32 accumulation of bf16 products
+@pytest.mark.parametrize("rows,dm,pitch", [(300, 192, None), (1000, 256, None), (129, 64, 128),
+                                           (128, 128, None), (517, 320, 512)])
+@pytest.mark.parametrize("dual", [True, False])
+def test_tensor_core_path_bf16(rows, dm, pitch, dual):
+    from paper_2604_00754_b200 import binding as sa
+    ya, yb, wa, wb = _draw(rows, dm, 3 + rows, torch.bfloat16, pitch)
+    args = [ya.cuda()[:, :dm], wa.cuda()]
+    if dual:
+        args += [yb.cuda()[:, :dm], wb.cuda()]
+    out = sa.sa_gate_projection_forward(*args)
+    assert sa.sa_read_status() == 0
+    _check(out, ya, wa, yb if dual else None, wb if dual else None, dm, 2e-2)
+
+
+@pytest.mark.parametrize("dtype,tol", [(torch.float32, 1e-4), (torch.bfloat16, 2e-2)])
+def test_plain_path_odd_sizes(dtype, tol):
+    from paper_2604_00754_b200 import binding as sa
+    rows, dm = 37, 50           # dm not a multiple of 64: the plain kernel
+    ya, yb, wa, wb = _draw(rows, dm, 5, dtype)
+    out = sa.sa_gate_projection_forward(ya.cuda(), wa.cuda(), yb.cuda(), wb.cuda())
+    assert sa.sa_read_status() == 0
+    _check(out, ya, wa, yb, wb, dm, tol)
+
+
+def test_model_width_sampled_rows():
+    """Qwen3-8B width (Hq*d = 4096) on the attention output layout [B,n,Hq,d] viewed as
+    [B*n, Hq*d]; sampled rows against the oracle."""
+    from paper_2604_00754_b200 import binding as sa
+    rows, dm = 4096, 4096
+    ya, yb, wa, wb = _draw(rows, dm, 9, torch.bfloat16)
+    out = sa.sa_gate_projection_forward(ya.cuda(), wa.cuda(), yb.cuda(), wb.cuda())
+    assert sa.sa_read_status() == 0
+    idx = torch.tensor([0, 1, 127, 128, 2047, 4095])
+    _check(out[idx.cuda()], ya[idx], wa, yb[idx], wb, dm, 2e-2)
+
+
+def test_rejects_bad_arguments():
+    from paper_2604_00754_b200 import binding as sa
+    y = torch.zeros(4, 64, dtype=torch.bfloat16, device="cuda")
+    w = torch.zeros(64, 32, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(ValueError):
+        sa.sa_gate_projection_forward(y, w)
