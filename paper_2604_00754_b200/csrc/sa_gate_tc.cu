@@ -22,7 +22,9 @@ namespace {
 constexpr int kBM = 128, kBN = 128, kBK = 64;
 constexpr int kStages = 3;
 constexpr int kTileBytes = 128 * kBK * 2;             // one 128 x 64 bf16 tile
-constexpr int kStageBytes = 4 * kTileBytes;           // Y_sa, W_sa, Y_swa, W_swa
+// a stage: Y_sa, W_sa, Y_swa, W_swa of one 64-wide K chunk, or, for the single path, Y, W of
+// two consecutive K chunks (so that one hand-over always feeds eight products)
+constexpr int kStageBytes = 4 * kTileBytes;
 constexpr int kGateThreads = 192;
 constexpr int kOffBars = kStages * kStageBytes;
 // barriers: full[kStages], empty[kStages], acc_full[2], acc_empty[2]
@@ -89,7 +91,6 @@ gate_tc_kernel(const __grid_constant__ GateParams p, const __grid_constant__ CUt
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   const int total = p.tiles_m * p.tiles_n;
-  const uint32_t stage_bytes = p.dual ? 4u * kTileBytes : 2u * kTileBytes;
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -104,13 +105,13 @@ gate_tc_kernel(const __grid_constant__ GateParams p, const __grid_constant__ CUt
             ok = mbar_wait(bar(kBarEmpty + s), (use / kStages - 1) & 1u, gave_up, p.status);
           if (!ok) break;
           const uint32_t dst = sbase + s * kStageBytes, fb = bar(kBarFull + s);
-          mbar_expect_tx(fb, stage_bytes);
-          tma_load_2d(dst, &tm_ysa, kc * kBK, m0, fb);
-          tma_load_2d(dst + kTileBytes, &tm_wsa, kc * kBK, n0, fb);
-          if (p.dual) {
-            tma_load_2d(dst + 2 * kTileBytes, &tm_yswa, kc * kBK, m0, fb);
-            tma_load_2d(dst + 3 * kTileBytes, &tm_wswa, kc * kBK, n0, fb);
-          }
+          mbar_expect_tx(fb, kStageBytes);
+          // single path: the second pair is the next K chunk (zeros past the last one)
+          const int k0 = (p.dual ? kc : 2 * kc) * kBK, k1 = p.dual ? k0 : k0 + kBK;
+          tma_load_2d(dst, &tm_ysa, k0, m0, fb);
+          tma_load_2d(dst + kTileBytes, &tm_wsa, k0, n0, fb);
+          tma_load_2d(dst + 2 * kTileBytes, &tm_yswa, k1, m0, fb);
+          tma_load_2d(dst + 3 * kTileBytes, &tm_wswa, k1, n0, fb);
         }
       }
       // Loads that were started but never consumed (only after a failed wait) must land
@@ -148,9 +149,9 @@ gate_tc_kernel(const __grid_constant__ GateParams p, const __grid_constant__ CUt
           const uint32_t lo = (sbase + s * kStageBytes) >> 4;
           mma_ss_x4(d_sa, desc64(lo | kLoK, kDescHi), desc64((lo + (kTileBytes >> 4)) | kLoK, kDescHi),
                     idesc, kc > 0);
-          if (p.dual)
-            mma_ss_x4(d_swa, desc64((lo + 2 * (kTileBytes >> 4)) | kLoK, kDescHi),
-                      desc64((lo + 3 * (kTileBytes >> 4)) | kLoK, kDescHi), idesc, kc > 0);
+          mma_ss_x4(p.dual ? d_swa : d_sa, desc64((lo + 2 * (kTileBytes >> 4)) | kLoK, kDescHi),
+                    desc64((lo + 3 * (kTileBytes >> 4)) | kLoK, kDescHi), idesc,
+                    p.dual ? (uint32_t)(kc > 0) : 1u);
           tc_commit(bar(kBarEmpty + s));      // the stage is free once these products are done
         }
         if (ok) tc_commit(bar(kBarAccFull + buf));
@@ -329,7 +330,7 @@ extern "C" sa_status sa_gate_projection_forward(int64_t rows, int32_t dm, int32_
     p.dm = dm; p.dual = y_swa != nullptr;
     p.tiles_m = (int)((rows + kBM - 1) / kBM);
     p.tiles_n = (dm + kBN - 1) / kBN;
-    p.k_chunks = dm / kBK;
+    p.k_chunks = p.dual ? dm / kBK : (dm / kBK + 1) / 2;    // hand-overs per tile
     p.status = status_ptr();
     if (!p.status) return SA_ERR_CUDA;
     if ((int64_t)p.tiles_m * p.tiles_n > 0x3fffffff) return SA_ERR_UNSUPPORTED;
