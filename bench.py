@@ -392,6 +392,28 @@ def extras(args, c, wl, sa, torch, dev, host, perm, inv, ws, y, pk):
         torch.cuda.empty_cache()
     res["table3_shape_B16_H16_d64_w256"] = t3
 
+    # projection gates of Eq. 5-6 at the workload's model width (Hq*d), all B*n tokens: two
+    # [B*n, dm] x [dm, dm] products on the tensor cores with the logistic and the combination
+    # of the two paths in the epilogue; random bf16 Y and W stand in for attention outputs
+    dm, rows_g = c.Hq * c.d, c.B * c.n
+    gg = torch.Generator(device="cuda").manual_seed(17)
+    ya = torch.randn(rows_g, dm, generator=gg, device="cuda").bfloat16()
+    yb = torch.randn(rows_g, dm, generator=gg, device="cuda").bfloat16()
+    wa = (torch.randn(dm, dm, generator=gg, device="cuda") * dm ** -0.5).bfloat16()
+    wb = (torch.randn(dm, dm, generator=gg, device="cuda") * dm ** -0.5).bfloat16()
+    og = torch.empty_like(ya)
+    g2 = event_ms(lambda: sa.sa_gate_projection_forward(ya, wa, yb, wb, out=og), it, 3, torch)
+    g1 = event_ms(lambda: sa.sa_gate_projection_forward(ya, wa, out=og), it, 3, torch)
+    gfl = 2.0 * rows_g * dm * dm
+    res["gate_projection"] = {
+        "rows": rows_g, "dm": dm,
+        "dual_ms": g2, "dual_tflops": 2 * gfl / (g2 * 1e-3) / 1e12,
+        "dual_frac_of_burst": 2 * gfl / (g2 * 1e-3) / 1e12 / pk["bf16_tflops"],
+        "single_ms": g1, "single_tflops": gfl / (g1 * 1e-3) / 1e12,
+        "single_frac_of_burst": gfl / (g1 * 1e-3) / 1e12 / pk["bf16_tflops"]}
+    del ya, yb, wa, wb, og
+    torch.cuda.empty_cache()
+
     rate, dt, rows, threads = oracle_sample_rate(c, host, 196608)
     res["cpu_baseline"] = {
         "value": rate, "unit": "tokens/s", "cores": threads, "kind": "oracle",
