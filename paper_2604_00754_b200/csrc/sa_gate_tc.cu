@@ -5,9 +5,10 @@
 // A dense contraction, so it runs on the 5th-generation tensor cores: a persistent grid of
 // one CTA per SM walks 128 x 128 output tiles.  Warp 0 streams 128 x 64 tiles of Y and of W
 // (both K-major, 128-byte swizzle) through a three-stage ring with TMA, warp 1 issues
-// tcgen05.mma into two fp32 accumulators per tile (one per path) in tensor memory, warps 2-5
+// tcgen05.mma into two fp32 accumulators per tile (one per path) in tensor memory, warps 2-9
 // read a finished pair of accumulators, apply the logistic, multiply by the rows of Y and
-// write the tile while the next tile's products already run into the other pair.
+// write the tile while the next tile's products already run into the other pair.  Tiles are
+// visited in blocks of 16 column tiles so that the slice of W in use stays in L2.
 //
 // Every mbarrier wait is bounded; on expiry the CTA records SA_ERR_TIMEOUT in the device
 // status word, stops issuing work, drains what it started and returns.
@@ -25,7 +26,7 @@ constexpr int kTileBytes = 128 * kBK * 2;             // one 128 x 64 bf16 tile
 // a stage: Y_sa, W_sa, Y_swa, W_swa of one 64-wide K chunk, or, for the single path, Y, W of
 // two consecutive K chunks (so that one hand-over always feeds eight products)
 constexpr int kStageBytes = 4 * kTileBytes;
-constexpr int kGateThreads = 192;
+constexpr int kGateThreads = 320;                    // TMA, MMA and eight epilogue warps
 constexpr int kOffBars = kStages * kStageBytes;
 // barriers: full[kStages], empty[kStages], acc_full[2], acc_empty[2]
 constexpr int kBarFull = 0, kBarEmpty = kStages, kBarAccFull = 2 * kStages,
@@ -56,7 +57,24 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm,
       : "memory");
 }
 
-__device__ __forceinline__ float logistic(float z) { return __frcp_rn(1.f + __expf(-z)); }
+// Tile order: blocks of kNB column tiles, inside a block row tile by row tile.  The CTAs that
+// run at the same time then share a slice of W that stays in L2 (kNB x 1 MB per path at
+// dm = 4096) while Y streams through once per block.
+constexpr int kNB = 16;
+__device__ __forceinline__ void tile_origin(const GateParams& p, int tile, int* m0, int* n0) {
+  const int per_block = p.tiles_m * kNB;
+  const int nb = tile / per_block, rem = tile - nb * per_block;
+  const int width = min(kNB, p.tiles_n - nb * kNB);
+  *m0 = (rem / width) * kBM;
+  *n0 = (nb * kNB + rem % width) * kBN;
+}
+
+// 1 / (1 + exp(-z)) = 0.5 tanh(z / 2) + 0.5: one special-function operation per element
+__device__ __forceinline__ float logistic(float z) {
+  float t;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(0.5f * z));
+  return fmaf(t, 0.5f, 0.5f);
+}
 
 __global__ void __launch_bounds__(kGateThreads, 1)
 gate_tc_kernel(const __grid_constant__ GateParams p, const __grid_constant__ CUtensorMap tm_ysa,
@@ -78,7 +96,7 @@ gate_tc_kernel(const __grid_constant__ GateParams p, const __grid_constant__ CUt
   if (threadIdx.x == 0) {
     *gave_up = 0;
     for (int i = 0; i < kNumBars; ++i)
-      mbar_init(bar(i), (i >= kBarAccEmpty) ? 128 : 1);
+      mbar_init(bar(i), (i >= kBarAccEmpty) ? 256 : 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -98,7 +116,8 @@ gate_tc_kernel(const __grid_constant__ GateParams p, const __grid_constant__ CUt
       uint32_t use = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < total && ok; tile += gridDim.x) {
-        const int m0 = (tile / p.tiles_n) * kBM, n0 = (tile % p.tiles_n) * kBN;
+        int m0, n0;
+        tile_origin(p, tile, &m0, &n0);
         for (int kc = 0; kc < p.k_chunks && ok; ++kc, ++use) {
           const uint32_t s = use % kStages;
           if (use >= (uint32_t)kStages)
@@ -159,15 +178,18 @@ gate_tc_kernel(const __grid_constant__ GateParams p, const __grid_constant__ CUt
     }
     __syncwarp();
   } else {
-    // ---------------------------------------------------------- epilogue (warps 2-5)
-    // A warp reads the 32 TMEM lanes 32 (warp % 4) .. +31: one output row per thread.
+    // ---------------------------------------------------------- epilogue (warps 2-9)
+    // A warp reads the 32 TMEM lanes 32 (warp % 4) .. +31: one output row per thread, and
+    // warps 2-5 take the first 64 columns of the tile, warps 6-9 the other 64.
+    const int half = (warp - 2) >> 2;
     const int row = (warp & 3) * 32 + lane;
     const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
     uint32_t it = 0;
     bool ok = true;
     for (int tile = blockIdx.x; tile < total; tile += gridDim.x, ++it) {
       const uint32_t buf = it & 1u;
-      const int m0 = (tile / p.tiles_n) * kBM, n0 = (tile % p.tiles_n) * kBN;
+      int m0, n0;
+      tile_origin(p, tile, &m0, &n0);
       ok = mbar_wait(bar(kBarAccFull + buf), (it / 2) & 1u, gave_up, p.status);
       ok = __all_sync(0xffffffffu, ok);       // the tensor-memory loads are warp-collective
       if (!ok) break;
@@ -178,7 +200,7 @@ gate_tc_kernel(const __grid_constant__ GateParams p, const __grid_constant__ CUt
       const __nv_bfloat16* yb = p.dual ? p.y_swa + r * p.ld_y + n0 : nullptr;
       __nv_bfloat16* o = p.out + r * p.ld_out + n0;
 #pragma unroll 1
-      for (int c = 0; c < kBN / 32; ++c) {
+      for (int c = 2 * half; c < 2 * half + 2; ++c) {
         uint32_t za[32], zb[32];
         tmem_ld32(tmem + lane_addr + buf * 256 + 32 * c, za);
         if (p.dual) tmem_ld32(tmem + lane_addr + buf * 256 + 128 + 32 * c, zb);
@@ -213,7 +235,7 @@ gate_tc_kernel(const __grid_constant__ GateParams p, const __grid_constant__ CUt
           }
         }
       }
-      // the accumulators may be overwritten once every thread of the four warps has read them
+      // the accumulators may be overwritten once every thread of the eight warps has read them
       tc_fence_before();
       mbar_arrive(bar(kBarAccEmpty + buf));
     }
