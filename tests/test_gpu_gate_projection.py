@@ -71,3 +71,39 @@ def test_rejects_bad_arguments():
     w = torch.zeros(64, 32, dtype=torch.bfloat16, device="cuda")
     with pytest.raises(ValueError):
         sa.sa_gate_projection_forward(y, w)
+
+
+def test_dual_path_block_on_token_major_layout():
+    """Alg. 2 with the projection gates of Eq. 6 end to end: Q/K/V stored token-major
+    ([B,n,H,d], as a QKV projection writes them), both attention branches write their outputs
+    in the same layout, and the gate product reads them as [B*n, Hq*d] without any copy."""
+    from paper_2604_00754_b200 import binding as sa
+    B, Hq, Hkv, n, d, w = 2, 4, 2, 700, 64, 256
+    dm = Hq * d
+    g = torch.Generator().manual_seed(21)
+    q = torch.randn(B, n, Hq, d, generator=g).bfloat16()
+    k = torch.randn(B, n, Hkv, d, generator=g).bfloat16()
+    v = torch.randn(B, n, Hkv, d, generator=g).bfloat16()
+    wa = (torch.randn(dm, dm, generator=g) * dm ** -0.5).bfloat16()
+    wb = (torch.randn(dm, dm, generator=g) * dm ** -0.5).bfloat16()
+    qd, kd, vd = (t.cuda().permute(0, 2, 1, 3) for t in (q, k, v))      # [B,H,n,d] views
+    perm, inv = sa.sa_make_perm(4, 0, B, n)
+    flags = sa.CAUSAL | sa.SWA_ONE_SIDED
+    y_sa = torch.empty(B, n, Hq, d, dtype=torch.bfloat16, device="cuda")
+    y_swa = torch.empty_like(y_sa)
+    sa.sa_forward(qd, kd, vd, perm, inv, w, flags, y=y_sa.permute(0, 2, 1, 3))
+    sa.sa_swa_forward(qd, kd, vd, w, flags, y=y_swa.permute(0, 2, 1, 3))
+    out = sa.sa_gate_projection_forward(y_sa.view(B * n, dm), wa.cuda(), y_swa.view(B * n, dm), wb.cuda())
+    assert sa.sa_read_status() == 0
+
+    f64 = lambda t: np.ascontiguousarray(t.permute(0, 2, 1, 3).double().numpy())
+    p_np, i_np = perm.cpu().numpy(), inv.cpu().numpy()
+    o_sa = oracle.sa_forward(f64(q), f64(k), f64(v), p_np, i_np, w, flags)[0]
+    o_swa = oracle.swa_forward(f64(q), f64(k), f64(v), w, flags)[0]
+    tok_major = lambda a: np.ascontiguousarray(a.transpose(0, 2, 1, 3)).reshape(B * n, dm)
+    want = oracle.gate_projection(tok_major(o_sa), wa.double().numpy(), tok_major(o_swa), wb.double().numpy())
+    got = out.double().cpu().numpy()
+    # two bf16 roundings in a row (branch outputs, then the gated sum) and a dm-long product
+    # of the rounded outputs: 3e-2 of max(|want|, 1)
+    err = np.abs(got - want) / np.maximum(np.abs(want), 1.0)
+    assert err.max() <= 3e-2, float(err.max())
