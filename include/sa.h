@@ -73,7 +73,8 @@ typedef enum {
   SA_OP_SWA_FORWARD = 2,
   SA_OP_GATED_FORWARD = 3,
   SA_OP_BACKWARD = 4,
-  SA_OP_COVERAGE = 5
+  SA_OP_COVERAGE = 5,
+  SA_OP_GATED_FORWARD_SCRATCH = 6 /* optional scratch of sa_swa_gated_forward, see there */
 } sa_op;
 
 typedef struct {
@@ -145,7 +146,11 @@ sa_status sa_swa_forward(const sa_problem* p, const void* q, const void* k, cons
 /* Gated SA + SWA forward (Alg. 2, Eq. 5) with per-head scalar gates:
  * y = sigmoid(gate_logits[0,hq]) * y_sa + sigmoid(gate_logits[1,hq]) * y_swa.
  * y: out.  y_sa, y_swa, lse_sa, lse_swa: out, nullable unless SA_SAVE_FOR_BWD; the
- * branch outputs are stored in the run dtype before they are combined. */
+ * branch outputs are stored in the run dtype before they are combined.
+ * ws is optional (sa_workspace_bytes(.., SA_OP_GATED_FORWARD) is 0).  When y_swa is given, or
+ * ws holds at least sa_workspace_bytes(.., SA_OP_GATED_FORWARD_SCRATCH) bytes (one branch
+ * output in q's layout), the branches run ungated and a streaming kernel combines them, which
+ * is faster; otherwise the SA branch's epilogue reads the local branch's rows and combines. */
 sa_status sa_swa_gated_forward(const sa_problem* p, const void* q, const void* k,
                                const void* v, const int32_t* perm, const int32_t* inv,
                                const float* gate_logits, void* y, void* y_sa, void* y_swa,

@@ -21,6 +21,7 @@ from . import build as _build
 SA_OK = 0
 CAUSAL, LINEAR_WINDOW, SWA_ONE_SIDED, SAVE_FOR_BWD, VALIDATE_PERM = 1, 2, 4, 8, 16
 OP_MAKE_PERM, OP_FORWARD, OP_SWA_FORWARD, OP_GATED_FORWARD, OP_BACKWARD, OP_COVERAGE = range(6)
+OP_GATED_FORWARD_SCRATCH = 6
 F32, BF16 = 0, 1
 
 EXPORTS = [
@@ -238,10 +239,13 @@ def sa_swa_forward(q, k, v, w, flags=CAUSAL | SWA_ONE_SIDED, scale=0.0, y=None, 
 
 
 def sa_swa_gated_forward(q, k, v, perm, inv, gate_logits, w, flags=CAUSAL | SWA_ONE_SIDED,
-                         scale=0.0, save_for_bwd=False, out=None):
+                         scale=0.0, save_for_bwd=False, out=None, ws=None, fused_epilogue=False):
     """Gated SA + SWA forward.  Returns y, or (y, y_sa, y_swa, lse_sa, lse_swa) when saving.
 
-    ``out`` may hold preallocated tensors under the keys y, y_sa, y_swa, lse_sa, lse_swa."""
+    ``out`` may hold preallocated tensors under the keys y, y_sa, y_swa, lse_sa, lse_swa.
+    ``ws``: optional scratch (uint8) for the local branch's rows when y_swa is not kept; one is
+    allocated when it is missing, unless ``fused_epilogue`` asks for the path that needs none
+    (the SA launch's epilogue then does the combination)."""
     lib = load_library()
     _same_layout(k, v)
     out = dict(out or {})
@@ -254,10 +258,18 @@ def sa_swa_gated_forward(q, k, v, perm, inv, gate_logits, w, flags=CAUSAL | SWA_
     y = out.setdefault("y", torch.empty_like(q))
     _same_layout(q, y, out.get("y_sa"), out.get("y_swa"))
     p = make_problem(q, k, w, flags, scale)
+    if fused_epilogue:
+        ws = None
+    elif ws is None and out.get("y_swa") is None:
+        # worth a scratch tensor and a third launch only when the outputs are large
+        nbytes = sa_workspace_bytes(p, OP_GATED_FORWARD_SCRATCH)
+        if nbytes >= (64 << 20):
+            ws = _workspace(nbytes, q.device, None)
     _check(lib.sa_swa_gated_forward(
         ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(perm), _ptr(inv), _ptr(gate_logits),
         _ptr(y), _ptr(out.get("y_sa")), _ptr(out.get("y_swa")), _ptr(out.get("lse_sa")),
-        _ptr(out.get("lse_swa")), None, 0, _stream()), "sa_swa_gated_forward")
+        _ptr(out.get("lse_swa")), _ptr(ws), 0 if ws is None else ws.numel(), _stream()),
+        "sa_swa_gated_forward")
     if save_for_bwd:
         return y, out["y_sa"], out["y_swa"], out["lse_sa"], out["lse_swa"]
     return y

@@ -52,6 +52,14 @@ sa_status check_problem(const sa_problem* p) {
   return SA_OK;
 }
 
+// Bytes of one branch output in the layout of q (its strides): what the gated forward can
+// use as scratch for the local branch's rows.
+size_t branch_bytes(const sa_problem* p) {
+  const int64_t elems = (p->B - 1) * p->q_stride[0] + (p->Hq - 1) * p->q_stride[1] +
+                        (int64_t)(p->n - 1) * p->q_stride[2] + p->d;
+  return (size_t)elems * (p->dtype == SA_BF16 ? 2 : 4);
+}
+
 float scale_of(const sa_problem* p) {
   return p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / std::sqrt((float)p->d);
 }
@@ -116,6 +124,8 @@ size_t sa_workspace_bytes(const sa_problem* p, int op) {
     case SA_OP_SWA_FORWARD:
     case SA_OP_GATED_FORWARD:
       return check_problem(p) == SA_OK ? 0 : (size_t)-1;
+    case SA_OP_GATED_FORWARD_SCRATCH:
+      return check_problem(p) == SA_OK ? branch_bytes(p) : (size_t)-1;
     case SA_OP_BACKWARD:
       if (check_problem(p) != SA_OK) return (size_t)-1;
       return bwd_ws_bytes(p->B, p->Hq, p->n, nullptr);
@@ -166,12 +176,12 @@ sa_status sa_swa_gated_forward(const sa_problem* p, const void* q, const void* k
                                const float* gate_logits, void* y, void* y_sa, void* y_swa,
                                float* lse_sa, float* lse_swa, void* ws, size_t ws_bytes,
                                sa_stream_t stream) {
-  (void)ws; (void)ws_bytes;
   sa_status s = check_problem(p);
   if (s != SA_OK) return s;
   if (!good_ptr(q) || !good_ptr(k) || !good_ptr(v) || !good_ptr(perm) || !good_ptr(inv) ||
       !good_ptr(y) || !gate_logits)
     return SA_ERR_INVALID_ARG;
+  if (ws && !aligned16(ws)) return SA_ERR_INVALID_ARG;
   if ((y_sa && !aligned16(y_sa)) || (y_swa && !aligned16(y_swa)) ||
       (lse_sa && !aligned16(lse_sa)) || (lse_swa && !aligned16(lse_swa)))
     return SA_ERR_INVALID_ARG;
@@ -179,7 +189,24 @@ sa_status sa_swa_gated_forward(const sa_problem* p, const void* q, const void* k
     return SA_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   if ((s = maybe_validate(p, perm, inv, st)) != SA_OK) return s;
-  // Local branch first: its rows land in y_swa (or in y itself when the caller does not keep
+  // With room for the local branch's rows (the caller's y_swa, or scratch) both branches run
+  // ungated and a streaming kernel combines them: cheaper than reading the other branch's
+  // row inside the attention epilogue, where the loads sit on the softmax warps' path.
+  void* swa_rows = y_swa ? y_swa : (ws && ws_bytes >= branch_bytes(p) ? ws : nullptr);
+  if (swa_rows) {
+    void* sa_rows = y_sa ? y_sa : y;
+    FwdArgs a = fwd_args(p, q, k, v, false);
+    a.perm = perm; a.inv = inv; a.y = sa_rows; a.lse = lse_sa;
+    cudaError_t e = run_forward(a, p->dtype, st);
+    if (e != cudaSuccess) return SA_ERR_CUDA;
+    FwdArgs b = fwd_args(p, q, k, v, true);
+    b.y = swa_rows; b.lse = lse_swa;
+    e = run_forward(b, p->dtype, st);
+    if (e != cudaSuccess) return SA_ERR_CUDA;
+    return from_cuda(launch_combine(y, sa_rows, swa_rows, gate_logits, p->B, p->Hq, p->n, p->d,
+                                    p->q_stride, p->dtype, st));
+  }
+  // Without it, local branch first: its rows land in y_swa (or in y itself when the caller does not keep
   // them).  The SA branch then owns each output row exactly once: it reads the local
   // branch's row, applies both gates and writes y.
   void* local_out = y_swa ? y_swa : y;

@@ -154,6 +154,10 @@ cudaError_t launch_fwd_simt(const FwdArgs& a, int dtype, cudaStream_t st);
 cudaError_t launch_validate_perm(const int32_t* perm, const int32_t* inv, int B, int n,
                                  cudaStream_t st);
 
+cudaError_t launch_combine(void* y, const void* y_sa, const void* y_swa, const float* logits,
+                           int B, int Hq, int n, int d, const int64_t s[3], int dtype,
+                           cudaStream_t st);
+
 cudaError_t launch_bwd_simt(const BwdArgs& a, int dtype, cudaStream_t st);
 size_t bwd_ws_bytes(int B, int Hq, int n, int* chunks_out);
 

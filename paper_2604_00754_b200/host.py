@@ -57,6 +57,9 @@ class HostForward:
         self.inv = torch.empty(B, n, dtype=torch.int32, device=dev)
         nbytes = sa.sa_workspace_bytes(sa.SaProblem(B=B, n=n), sa.OP_MAKE_PERM)
         self.ws = torch.empty(max(nbytes, 1), dtype=torch.uint8, device=dev)
+        # scratch for the local branch's rows of one head group (in the layout of y)
+        self.scratch = torch.empty(self.y.numel() * self.y.element_size(), dtype=torch.uint8,
+                                   device=dev)
         self.s_in = torch.cuda.Stream(dev)
         self.s_run = torch.cuda.Stream(dev)
         self.s_out = torch.cuda.Stream(dev)
@@ -95,7 +98,7 @@ class HostForward:
                 self.gate_g[i].copy_(self.gate[:, qa:qb])
                 sa.sa_swa_gated_forward(self.q[:, qa:qb], self.k[:, ka:kb], self.v[:, ka:kb],
                                         self.perm, self.inv, self.gate_g[i], self.w, self.flags,
-                                        out={"y": self.y[:, qa:qb]})
+                                        out={"y": self.y[:, qa:qb]}, ws=self.scratch)
                 self.ev_done[i].record(self.s_run)
         with torch.cuda.stream(self.s_out):
             for i, (_, _, qa, qb) in enumerate(self.groups):

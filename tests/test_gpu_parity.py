@@ -263,6 +263,31 @@ def test_gated_forward_small(dtype, save):
         close(out, ref[0], dtype, "y")
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("fused", [False, True])
+@pytest.mark.parametrize("token_major", [False, True])
+def test_gated_forward_both_combine_paths(dtype, fused, token_major):
+    """The gates are applied either by a streaming kernel over both branch outputs (scratch
+    given) or inside the SA launch's epilogue (no scratch); d = 128 and w = 300 put the bf16
+    case on the tensor-core kernels with 128-key blocks.  Also on token-major tensors."""
+    B, Hq, Hkv, n, d, w = 1, 4, 2, 521, 128, 300
+    flags = CAUSAL | SWA_ONE_SIDED
+    q, k, v = draw((B, Hq, n, d), (B, Hkv, n, d), dtype, seed=31)
+    lg = torch.randn(2, Hq, generator=torch.Generator().manual_seed(6))
+    perm, inv, permc, invc = perms(31, 1, B, n)
+    if token_major:   # memory order [B,n,H,d], seen as [B,H,n,d]
+        dev = [t.permute(0, 2, 1, 3).contiguous().cuda().permute(0, 2, 1, 3) for t in (q, k, v)]
+    else:
+        dev = [t.cuda() for t in (q, k, v)]
+    y = torch.empty_like(dev[0])
+    sa.sa_swa_gated_forward(dev[0], dev[1], dev[2], perm, inv, lg.cuda(), w, flags,
+                            out={"y": y}, fused_epilogue=fused)
+    assert sa.sa_read_status() == 0
+    ref = oracle.gated_forward(as_f64(q), as_f64(k), as_f64(v), permc, invc, lg.double().numpy(),
+                               w, flags)
+    close(y, ref[0], dtype, "y")
+
+
 # --------------------------------------------------------------------- backward
 
 def run_backward(q, k, v, dy, lg, perm, inv, w, flags):
