@@ -280,8 +280,16 @@ def test_gated_forward_both_combine_paths(dtype, fused, token_major):
     else:
         dev = [t.cuda() for t in (q, k, v)]
     y = torch.empty_like(dev[0])
+    ws = None
+    if not fused:
+        nbytes = sa.sa_workspace_bytes(sa.make_problem(dev[0], dev[1], w, flags),
+                                       sa.OP_GATED_FORWARD_SCRATCH)
+        assert nbytes >= y.numel() * y.element_size()
+        ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    launches = sa.launch_count()
     sa.sa_swa_gated_forward(dev[0], dev[1], dev[2], perm, inv, lg.cuda(), w, flags,
-                            out={"y": y}, fused_epilogue=fused)
+                            out={"y": y}, ws=ws, fused_epilogue=fused)
+    assert sa.launch_count() - launches == (2 if fused else 3)
     assert sa.sa_read_status() == 0
     ref = oracle.gated_forward(as_f64(q), as_f64(k), as_f64(v), permc, invc, lg.double().numpy(),
                                w, flags)
