@@ -192,8 +192,12 @@ sa_status sa_swa_gated_forward(const sa_problem* p, const void* q, const void* k
   // With room for the local branch's rows (the caller's y_swa, or scratch) both branches run
   // ungated and a streaming kernel combines them: cheaper than reading the other branch's
   // row inside the attention epilogue, where the loads sit on the softmax warps' path.
-  void* swa_rows = y_swa ? y_swa : (ws && ws_bytes >= branch_bytes(p) ? ws : nullptr);
-  if (swa_rows) {
+  // Scratch says the caller wants this path; with only y_swa to go by it is taken for large
+  // outputs (measured: from about 64 MB per branch the third launch costs less than the
+  // epilogue loads; below, e.g. the 50 MB of the pre-training shape, it does not).
+  const bool scratch = ws && ws_bytes >= branch_bytes(p);
+  void* swa_rows = y_swa ? y_swa : (scratch ? ws : nullptr);
+  if (swa_rows && (scratch || branch_bytes(p) >= ((size_t)64 << 20))) {
     void* sa_rows = y_sa ? y_sa : y;
     FwdArgs a = fwd_args(p, q, k, v, false);
     a.perm = perm; a.inv = inv; a.y = sa_rows; a.lse = lse_sa;

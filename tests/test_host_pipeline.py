@@ -41,12 +41,15 @@ def test_pipelined_forward_equals_single_call(n_groups):
     hf.forward(q, k, v, lg, hy, seed=5, layer=2)
     torch.cuda.synchronize()
     perm, inv = sa.sa_make_perm(5, 2, B, n)
-    ref = sa.sa_swa_gated_forward(q.cuda(), k.cuda(), v.cuda(), perm, inv, lg.cuda(), w)
+    # the pipeline hands the library scratch, so its gates are applied by the streaming
+    # kernel: the single call does the same (the fused epilogue rounds differently)
+    scratch = torch.empty(hy.numel() * hy.element_size(), dtype=torch.uint8, device="cuda")
+    ref = sa.sa_swa_gated_forward(q.cuda(), k.cuda(), v.cuda(), perm, inv, lg.cuda(), w, ws=scratch)
     assert sa.sa_read_status() == 0
     assert torch.equal(hy, ref.cpu())
     # a second call with another layer index draws another permutation
     hf.forward(q, k, v, lg, hy, seed=5, layer=3)
     torch.cuda.synchronize()
     perm, inv = sa.sa_make_perm(5, 3, B, n)
-    ref = sa.sa_swa_gated_forward(q.cuda(), k.cuda(), v.cuda(), perm, inv, lg.cuda(), w)
+    ref = sa.sa_swa_gated_forward(q.cuda(), k.cuda(), v.cuda(), perm, inv, lg.cuda(), w, ws=scratch)
     assert torch.equal(hy, ref.cpu())
