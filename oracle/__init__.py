@@ -267,3 +267,26 @@ def gate_projection(y_sa, w_sa, y_swa=None, w_swa=None):
     if y_swa is not None:
         out = out + one(y_swa, w_swa)
     return out
+
+
+def gate_projection_backward(dout, y_sa, w_sa, y_swa=None, w_swa=None):
+    """Derivative of gate_projection (Eq. 5-6) with respect to its inputs and weights.
+
+    With z = y w^T and g = sigmoid(z), out = g * y per path, so for an upstream gradient dout
+        dz = dout * y * g * (1 - g),   dw = dz^T y,   dy = dout * g + dz w.
+    Returns (dy_sa, dw_sa) for the single path, (dy_sa, dw_sa, dy_swa, dw_swa) for the dual
+    path (the paths only share dout).  Plain float64 numpy."""
+    dout = np.asarray(dout, dtype=np.float64)
+
+    def one(y, w):
+        y = np.asarray(y, dtype=np.float64)
+        w = np.asarray(w, dtype=np.float64)
+        if y.ndim != 2 or w.shape != (y.shape[1], y.shape[1]) or dout.shape != y.shape:
+            raise ValueError("y and dout must be [rows, dm] and w [dm, dm]")
+        g = 1.0 / (1.0 + np.exp(-(y @ w.T)))
+        dz = dout * y * g * (1.0 - g)
+        return dout * g + dz @ w, dz.T @ y
+    res = one(y_sa, w_sa)
+    if y_swa is not None:
+        res = res + one(y_swa, w_swa)
+    return res

@@ -67,3 +67,45 @@ def test_paths_are_independent_and_saturate():
 def test_shape_errors():
     with pytest.raises(ValueError):
         oracle.gate_projection(np.zeros((2, 3)), np.zeros((3, 4)))
+
+
+def _loss(ya, wa, yb, wb, c):
+    return float((oracle.gate_projection(ya, wa, yb, wb) * c).sum())
+
+
+def test_backward_matches_central_differences_of_the_forward():
+    # the forward oracle is pinned above; its numerical derivative pins the backward
+    r = _rng(4)
+    ya, yb = r.standard_normal((3, 4)), r.standard_normal((3, 4))
+    wa, wb = r.standard_normal((4, 4)), r.standard_normal((4, 4))
+    c = r.standard_normal((3, 4))              # upstream gradient: loss = sum(out * c)
+    dya, dwa, dyb, dwb = oracle.gate_projection_backward(c, ya, wa, yb, wb)
+    eps = 1e-6
+    for arr, grad, which in ((ya, dya, 0), (wa, dwa, 1), (yb, dyb, 2), (wb, dwb, 3)):
+        num = np.zeros_like(arr)
+        for idx in np.ndindex(arr.shape):
+            args = [ya.copy(), wa.copy(), yb.copy(), wb.copy()]
+            args[which][idx] += eps
+            up = _loss(*args, c)
+            args[which][idx] -= 2 * eps
+            num[idx] = (up - _loss(*args, c)) / (2 * eps)
+        np.testing.assert_allclose(grad, num, rtol=1e-6, atol=1e-8)
+
+
+def test_backward_zero_weights_closed_form():
+    # w = 0: g = 1/2 everywhere, dz = dout * y / 4, so dy = dout / 2 and dw = (dout * y)^T y / 4
+    r = _rng(5)
+    y, c = r.standard_normal((5, 3)), r.standard_normal((5, 3))
+    dy, dw = oracle.gate_projection_backward(c, y, np.zeros((3, 3)))
+    np.testing.assert_allclose(dy, 0.5 * c, rtol=0, atol=1e-15)
+    np.testing.assert_allclose(dw, (c * y).T @ y / 4.0, rtol=1e-14)
+
+
+def test_backward_single_path_is_the_dual_path_with_a_dead_branch():
+    r = _rng(6)
+    y, c, w = r.standard_normal((4, 3)), r.standard_normal((4, 3)), r.standard_normal((3, 3))
+    dy1, dw1 = oracle.gate_projection_backward(c, y, w)
+    dy2, dw2, dyb, dwb = oracle.gate_projection_backward(c, y, w, np.zeros((4, 3)), w)
+    np.testing.assert_allclose(dy1, dy2, rtol=0, atol=0)
+    np.testing.assert_allclose(dw1, dw2, rtol=0, atol=0)
+    np.testing.assert_allclose(dwb, 0 * dwb, atol=0)
