@@ -198,6 +198,25 @@ sa_status sa_gate_projection_forward(int64_t rows, int32_t dm, int32_t dtype, co
                                      const void* w_swa, void* out, int64_t ld_out,
                                      sa_stream_t stream);
 
+/* Backward of sa_gate_projection_forward.  With z = y w^T, g = sigmoid(z) per path:
+ *   dz = dout * y * g * (1 - g),   dw = dz^T y,   dy = dout * g + dz w.
+ * dout: device, [rows, dm], pitch ld_dout: gradient of the forward's out.  y_*, w_*: as in the
+ * forward (y pitch ld_y).  dy_sa, dy_swa: out, [rows, dm], pitch ld_dy; dw_sa, dw_swa: out,
+ * [dm, dm] contiguous, the sum over all rows (not accumulated into).  y_swa == NULL: single
+ * path, the swa arguments are ignored.  ws: device scratch of
+ * sa_gate_projection_backward_ws_bytes(rows, dm) bytes (dz and dout * g of one path at a
+ * time).  bf16 with dm a multiple of 64 and 16-byte aligned rows runs three tensor-core
+ * products per path (dz and dout * g are kept in bf16 between them); every other case runs
+ * plain kernels with fp32 scratch.  Nothing is allocated; outputs may not alias inputs.
+ * Errors: SA_ERR_INVALID_ARG, SA_ERR_WORKSPACE, SA_ERR_UNSUPPORTED, SA_ERR_CUDA. */
+size_t sa_gate_projection_backward_ws_bytes(int64_t rows, int32_t dm);
+sa_status sa_gate_projection_backward(int64_t rows, int32_t dm, int32_t dtype, const void* dout,
+                                      int64_t ld_dout, const void* y_sa, const void* y_swa,
+                                      int64_t ld_y, const void* w_sa, const void* w_swa,
+                                      void* dy_sa, void* dy_swa, int64_t ld_dy, void* dw_sa,
+                                      void* dw_swa, void* ws, size_t ws_bytes,
+                                      sa_stream_t stream);
+
 /* Synchronises the stream, returns the device status word (SA_OK, SA_ERR_BAD_PERM or
  * SA_ERR_TIMEOUT) of the current device and clears it. */
 sa_status sa_read_status(sa_stream_t stream);

@@ -28,7 +28,8 @@ EXPORTS = [
     "sa_problem_set_contiguous", "sa_workspace_bytes", "sa_make_perm", "sa_forward",
     "sa_swa_forward", "sa_swa_gated_forward", "sa_backward", "sa_coverage", "sa_read_status",
     "sa_status_string", "sa_launch_count", "sa_set_profile_events", "sa_make_perm_static",
-    "sa_gate_projection_forward",
+    "sa_gate_projection_forward", "sa_gate_projection_backward",
+    "sa_gate_projection_backward_ws_bytes",
 ]
 
 
@@ -84,6 +85,12 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.sa_gate_projection_forward.argtypes = [ctypes.c_int64, i32, i32, vp, vp, ctypes.c_int64,
                                                vp, vp, vp, ctypes.c_int64, vp]
     lib.sa_gate_projection_forward.restype = ctypes.c_int
+    i64 = ctypes.c_int64
+    lib.sa_gate_projection_backward_ws_bytes.argtypes = [i64, i32]
+    lib.sa_gate_projection_backward_ws_bytes.restype = sz
+    lib.sa_gate_projection_backward.argtypes = [i64, i32, i32, vp, i64, vp, vp, i64, vp, vp, vp, vp,
+                                                i64, vp, vp, vp, sz, vp]
+    lib.sa_gate_projection_backward.restype = ctypes.c_int
     lib.sa_read_status.argtypes = [vp]
     for f in ("sa_make_perm", "sa_forward", "sa_swa_forward", "sa_swa_gated_forward",
               "sa_backward", "sa_coverage", "sa_read_status"):
@@ -345,6 +352,36 @@ def sa_gate_projection_forward(y_sa, w_sa, y_swa=None, w_swa=None, out=None):
                                           _ptr(w_sa), _ptr(w_swa), _ptr(out), out.stride(0),
                                           _stream()), "sa_gate_projection_forward")
     return out
+
+
+def sa_gate_projection_backward(dout, y_sa, w_sa, y_swa=None, w_swa=None, ws=None):
+    """Gradients of sa_gate_projection_forward: (dy_sa, dw_sa) or, for the dual path,
+    (dy_sa, dw_sa, dy_swa, dw_swa).  Tensors as in the forward; dout: [rows, dm]."""
+    lib = load_library()
+    rows, dm = y_sa.shape
+    dt = {torch.float32: 0, torch.bfloat16: 1}.get(y_sa.dtype)
+    if dt is None:
+        raise ValueError("dtype must be float32 or bfloat16")
+    for t in (dout, y_sa, y_swa):
+        if t is not None and (t.dim() != 2 or t.stride(1) != 1 or t.shape != y_sa.shape
+                              or t.dtype != y_sa.dtype):
+            raise ValueError("dout and y tensors must be [rows, dm] with unit inner stride")
+    if y_swa is not None and y_swa.stride(0) != y_sa.stride(0):
+        raise ValueError("y_sa and y_swa must share one row pitch")
+    for t in (w_sa, w_swa):
+        if t is not None and (tuple(t.shape) != (dm, dm) or not t.is_contiguous()
+                              or t.dtype != y_sa.dtype):
+            raise ValueError("w tensors must be contiguous [dm, dm] of the run dtype")
+    dual = y_swa is not None
+    dy_sa, dw_sa = torch.empty_like(y_sa, memory_format=torch.contiguous_format), torch.empty_like(w_sa)
+    dy_swa = torch.empty_like(dy_sa) if dual else None
+    dw_swa = torch.empty_like(w_sa) if dual else None
+    ws = _workspace(int(lib.sa_gate_projection_backward_ws_bytes(rows, dm)), y_sa.device, ws)
+    _check(lib.sa_gate_projection_backward(
+        rows, dm, dt, _ptr(dout), dout.stride(0), _ptr(y_sa), _ptr(y_swa), y_sa.stride(0),
+        _ptr(w_sa), _ptr(w_swa), _ptr(dy_sa), _ptr(dy_swa), dy_sa.stride(0), _ptr(dw_sa),
+        _ptr(dw_swa), _ptr(ws), ws.numel(), _stream()), "sa_gate_projection_backward")
+    return (dy_sa, dw_sa, dy_swa, dw_swa) if dual else (dy_sa, dw_sa)
 
 
 def sa_read_status() -> int:

@@ -107,3 +107,44 @@ def test_dual_path_block_on_token_major_layout():
     # of the rounded outputs: 3e-2 of max(|want|, 1)
     err = np.abs(got - want) / np.maximum(np.abs(want), 1.0)
     assert err.max() <= 3e-2, float(err.max())
+
+
+def _check_grads(got, want, tol):
+    for g, w_, name in zip(got, want, ("dy_sa", "dw_sa", "dy_swa", "dw_swa")):
+        g = g.double().cpu().numpy()
+        # gradients are sums of many signed terms: the bound is relative to the tensor's scale
+        scale = max(np.abs(w_).max(), 1e-6)
+        err = np.abs(g - w_).max() / scale
+        assert err <= tol, (name, float(err))
+
+
+@pytest.mark.parametrize("rows,dm,pitch", [(300, 192, None), (1000, 256, None), (129, 64, 128),
+                                           (128, 128, None), (517, 320, 512)])
+@pytest.mark.parametrize("dual", [True, False])
+def test_backward_tensor_core_path_bf16(rows, dm, pitch, dual):
+    from paper_2604_00754_b200 import binding as sa
+    ya, yb, wa, wb = _draw(rows, dm, 13 + rows, torch.bfloat16, pitch)
+    dout = torch.randn(rows, dm, generator=torch.Generator().manual_seed(rows)).bfloat16()
+    args = [dout.cuda(), ya.cuda()[:, :dm], wa.cuda()]
+    if dual:
+        args += [yb.cuda()[:, :dm], wb.cuda()]
+    got = sa.sa_gate_projection_backward(*args)
+    assert sa.sa_read_status() == 0
+    want = oracle.gate_projection_backward(
+        dout.double().numpy(), ya[:, :dm].double().numpy(), wa.double().numpy(),
+        yb[:, :dm].double().numpy() if dual else None, wb.double().numpy() if dual else None)
+    # bf16 intermediates (dz, dout * g) and bf16 results, fp32 accumulation: 2e-2 of the scale
+    _check_grads(got, want, 2e-2)
+
+
+@pytest.mark.parametrize("dtype,tol", [(torch.float32, 1e-4), (torch.bfloat16, 2e-2)])
+def test_backward_plain_path_odd_sizes(dtype, tol):
+    from paper_2604_00754_b200 import binding as sa
+    rows, dm = 37, 50
+    ya, yb, wa, wb = _draw(rows, dm, 15, dtype)
+    dout = torch.randn(rows, dm, generator=torch.Generator().manual_seed(2)).to(dtype)
+    got = sa.sa_gate_projection_backward(dout.cuda(), ya.cuda(), wa.cuda(), yb.cuda(), wb.cuda())
+    assert sa.sa_read_status() == 0
+    want = oracle.gate_projection_backward(dout.double().numpy(), ya.double().numpy(), wa.double().numpy(),
+                                           yb.double().numpy(), wb.double().numpy())
+    _check_grads(got, want, tol)
