@@ -415,7 +415,13 @@ def extras(args, c, wl, sa, torch, dev, host, perm, inv, ws, y, pk):
         "dual_frac_of_burst": 2 * gfl / (g2 * 1e-3) / 1e12 / pk["bf16_tflops"],
         "single_ms": g1, "single_tflops": gfl / (g1 * 1e-3) / 1e12,
         "single_frac_of_burst": gfl / (g1 * 1e-3) / 1e12 / pk["bf16_tflops"]}
-    del ya, yb, wa, wb, og
+    # and their backward (dz, dy, dw: three products per path)
+    gbw = torch.empty(rows_g * dm * 8, dtype=torch.uint8, device="cuda")
+    gb2 = event_ms(lambda: sa.sa_gate_projection_backward(og, ya, wa, yb, wb, ws=gbw), 3, 2, torch)
+    res["gate_projection"].update({
+        "bwd_dual_ms": gb2, "bwd_dual_tflops": 6 * gfl / (gb2 * 1e-3) / 1e12,
+        "bwd_dual_frac_of_burst": 6 * gfl / (gb2 * 1e-3) / 1e12 / pk["bf16_tflops"]})
+    del ya, yb, wa, wb, og, gbw
     torch.cuda.empty_cache()
 
     rate, dt, rows, threads = oracle_sample_rate(c, host, 196608)
