@@ -375,6 +375,7 @@ def extras(args, c, wl, sa, torch, dev, host, perm, inv, ws, y, pk):
     # forward + backward of single-path SA); the paper's A100 / FlexAttention times are context
     t3 = {}
     paper_ms = {2048: 5.4, 4096: 7.9, 8192: 15.2, 16384: 29.6, 32768: 52.8}
+    paper_full_ms = {2048: 8.0, 4096: 27.2, 8192: 99.7, 16384: 379.9, 32768: 1477.0}
     for n3 in (2048, 8192, 32768):
         c3 = wl.Workload("table3", "bf16", 16, 16, 16, n3, 64, 256, seed=9, ops="gated_fwd_bwd")
         d3 = {k_: v_.cuda() for k_, v_ in wl.draw(c3).items()}
@@ -392,6 +393,18 @@ def extras(args, c, wl, sa, torch, dev, host, perm, inv, ws, y, pk):
             o3.update(zip(("dq", "dk", "dv", "dgate"), r))
         t3[str(n3)] = {"sa_fwd_bwd_ms": event_ms(fb3, 3, 2, torch),
                        "paper_a100_flexattention_ms": paper_ms[n3]}
+        # the table's other column: full causal attention, here the same kernels with the
+        # identity permutation and a window that covers the whole sequence
+        ident = torch.arange(c3.n, dtype=torch.int32, device="cuda").repeat(c3.B, 1).contiguous()
+        wfull = 2 * c3.n + 1
+
+        def full3():
+            sa.sa_forward(d3["q"], d3["k"], d3["v"], ident, ident, wfull, sa.CAUSAL, y=y3, lse=l3)
+            r = sa.sa_backward(d3["q"], d3["k"], d3["v"], ident, ident, None, y3, None, l3, None,
+                               d3["dy"], wfull, sa.CAUSAL, ws=w3, out=o3)
+            o3.update(zip(("dq", "dk", "dv", "dgate"), r))
+        t3[str(n3)]["full_attention_fwd_bwd_ms"] = event_ms(full3, 2, 1, torch)
+        t3[str(n3)]["paper_a100_full_attention_ms"] = paper_full_ms[n3]
         del d3, y3, l3, w3, o3
         torch.cuda.empty_cache()
     res["table3_shape_B16_H16_d64_w256"] = t3
