@@ -148,3 +148,15 @@ def test_backward_plain_path_odd_sizes(dtype, tol):
     want = oracle.gate_projection_backward(dout.double().numpy(), ya.double().numpy(), wa.double().numpy(),
                                            yb.double().numpy(), wb.double().numpy())
     _check_grads(got, want, tol)
+
+
+def test_backward_model_width_single_path():
+    """Qwen3-8B width (dm = 4096), 4096 tokens, single path, whole result against the oracle."""
+    from paper_2604_00754_b200 import binding as sa
+    rows, dm = 4096, 4096
+    ya, _, wa, _ = _draw(rows, dm, 19, torch.bfloat16)
+    dout = torch.randn(rows, dm, generator=torch.Generator().manual_seed(3)).bfloat16()
+    got = sa.sa_gate_projection_backward(dout.cuda(), ya.cuda(), wa.cuda())
+    assert sa.sa_read_status() == 0
+    want = oracle.gate_projection_backward(dout.double().numpy(), ya.double().numpy(), wa.double().numpy())
+    _check_grads(got, want, 2e-2)
