@@ -12,10 +12,7 @@
 //
 // Every mbarrier wait is bounded; on expiry the CTA records SA_ERR_TIMEOUT in the device
 // status word, stops issuing work, drains what it started and returns.
-#include <cuda.h>
-
-#include "sa_common.cuh"
-#include "sa_tc_common.cuh"
+#include "sa_gemm_common.cuh"
 
 namespace sa {
 namespace {
@@ -44,18 +41,6 @@ struct BwdGateParams {
   int* status;
 };
 
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
-               : "memory");
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y,
-                                            uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes "
-      "[%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(bar)
-      : "memory");
-}
 __device__ __forceinline__ void mma_ss(uint32_t d, uint64_t a, uint64_t b, uint32_t idesc,
                                        uint32_t acc) {
   asm volatile(
@@ -68,12 +53,6 @@ __device__ __forceinline__ void mma_ss(uint32_t d, uint64_t a, uint64_t b, uint3
 __host__ __device__ constexpr uint32_t idesc_of(bool a_mn, bool b_mn) {
   return instr_desc(kT, kT, b_mn) | ((a_mn ? 1u : 0u) << 15);
 }
-__device__ __forceinline__ float logistic(float z) {
-  float t;
-  asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(0.5f * z));
-  return fmaf(t, 0.5f, 0.5f);
-}
-
 template <int MODE>
 __global__ void __launch_bounds__(kThreadsB, 1)
 gate_bwd_kernel(const __grid_constant__ BwdGateParams p, const __grid_constant__ CUtensorMap tm_a,
@@ -321,43 +300,6 @@ __global__ void dw_simt_kernel(int64_t rows, int dm, const float* __restrict__ d
 }
 
 // ------------------------------------------------------------------------------ host
-
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
-                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
-                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
-    void* ptr = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) ==
-            cudaSuccess && qres == cudaDriverEntryPointSuccess)
-      fn = (EncodeTiledFn)ptr;
-  }
-  return fn;
-}
-
-// bf16 matrix [rows, cols], pitch ld elements, read in boxes of 64 columns x box_rows rows
-// with the 128-byte swizzle; outside the matrix reads zero.  box_rows 128: an operand whose
-// columns are the contraction index; 64: one whose rows are.
-bool make_map(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int64_t ld,
-              int box_rows) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
-  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-  const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
-  const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
-  const cuuint32_t estr[2] = {1, 1};
-  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
-            estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
 
 template <int MODE>
 cudaError_t launch_mode(BwdGateParams p, const CUtensorMap& a, const CUtensorMap& b, int64_t k,

@@ -12,10 +12,7 @@
 //
 // Every mbarrier wait is bounded; on expiry the CTA records SA_ERR_TIMEOUT in the device
 // status word, stops issuing work, drains what it started and returns.
-#include <cuda.h>
-
-#include "sa_common.cuh"
-#include "sa_tc_common.cuh"
+#include "sa_gemm_common.cuh"
 
 namespace sa {
 namespace {
@@ -43,20 +40,6 @@ struct GateParams {
   int* status;
 };
 
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
-               : "memory");
-}
-// One 64 x 128 box (x: element column, a multiple of 64; y: row) into shared memory.
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y,
-                                            uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes "
-      "[%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"(tm), "r"(x), "r"(y), "r"(bar)
-      : "memory");
-}
-
 // Tile order: blocks of kNB column tiles, inside a block row tile by row tile.  The CTAs that
 // run at the same time then share a slice of W that stays in L2 (kNB x 1 MB per path at
 // dm = 4096) while Y streams through once per block.
@@ -67,13 +50,6 @@ __device__ __forceinline__ void tile_origin(const GateParams& p, int tile, int* 
   const int width = min(kNB, p.tiles_n - nb * kNB);
   *m0 = (rem / width) * kBM;
   *n0 = (nb * kNB + rem % width) * kBN;
-}
-
-// 1 / (1 + exp(-z)) = 0.5 tanh(z / 2) + 0.5: one special-function operation per element
-__device__ __forceinline__ float logistic(float z) {
-  float t;
-  asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(0.5f * z));
-  return fmaf(t, 0.5f, 0.5f);
 }
 
 __global__ void __launch_bounds__(kGateThreads, 1)
@@ -280,41 +256,6 @@ __global__ void gate_simt_kernel(int64_t rows, int dm, const T* __restrict__ y_s
   out[r * ld_out + o] = from_f32<T>(acc);
 }
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
-                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
-                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
-    void* ptr = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) ==
-            cudaSuccess && qres == cudaDriverEntryPointSuccess)
-      fn = (EncodeTiledFn)ptr;
-  }
-  return fn;
-}
-
-// bf16 matrix [rows, cols] with row pitch ld (elements), read in boxes of 64 columns x 128
-// rows laid out with the 128-byte swizzle; rows and columns past the end read as zero.
-bool make_map(CUtensorMap* tm, const void* base, int64_t rows, int64_t cols, int64_t ld) {
-  EncodeTiledFn fn = encode_fn();
-  if (!fn) return false;
-  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-  const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
-  const cuuint32_t box[2] = {(cuuint32_t)kBK, 128};
-  const cuuint32_t estr[2] = {1, 1};
-  return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
-            estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-bool aligned16(const void* p) { return ((uintptr_t)p & 15u) == 0; }
-
 }  // namespace
 }  // namespace sa
 
@@ -341,8 +282,8 @@ extern "C" sa_status sa_gate_projection_forward(int64_t rows, int32_t dm, int32_
     CUtensorMap tm[4];
     const void* ysw = y_swa ? y_swa : y_sa;      // unused maps still have to be valid
     const void* wsw = y_swa ? w_swa : w_sa;
-    if (!make_map(&tm[0], y_sa, rows, dm, ld_y) || !make_map(&tm[1], w_sa, dm, dm, dm) ||
-        !make_map(&tm[2], ysw, rows, dm, ld_y) || !make_map(&tm[3], wsw, dm, dm, dm))
+    if (!make_map(&tm[0], y_sa, rows, dm, ld_y, 128) || !make_map(&tm[1], w_sa, dm, dm, dm, 128) ||
+        !make_map(&tm[2], ysw, rows, dm, ld_y, 128) || !make_map(&tm[3], wsw, dm, dm, dm, 128))
       return SA_ERR_CUDA;
     GateParams p{};
     p.y_sa = (const __nv_bfloat16*)y_sa;
