@@ -14,7 +14,9 @@
 // of Eq. 5 when asked, and scatters each row to its original position.
 //
 // Warp roles (384 threads): warp 0 MMA issuer and TMEM allocator, warps 1-3 gather
-// producers, warps 4-7 softmax/epilogue of query tile 0, warps 8-11 of query tile 1.
+// producers (for the one-sided SWA branch, whose rows are consecutive, one thread that loads
+// whole tiles by TMA instead), warps 4-7 softmax/epilogue of query tile 0, warps 8-11 of
+// query tile 1.
 // While one tile's softmax runs, the tensor core works on the other tile.  K and V tiles
 // travel through one ring of shared-memory slots (K0 V0 K1 V1 ...), and every barrier is
 // addressed by counters that run on across items, so the loads, products and epilogue of
@@ -25,6 +27,7 @@
 #include <type_traits>
 
 #include "sa_fwd_tc.cuh"
+#include "sa_gemm_common.cuh"
 #include "sa_tc_common.cuh"
 
 namespace sa {
@@ -49,6 +52,10 @@ struct TcParams {
   const int* abort_flag;
   int B, Hq, Hkv, G, n, w, h;
   int causal, linear, one_sided, swa, full_range;
+  // One-sided SWA branch on tensors that are plain 2-D matrices of rows: whole tiles come
+  // by TMA (row of (b, h, token) = b * rb + h * rh + token, first column h * ch)
+  int use_tma;
+  int64_t q_rb, q_rh, q_ch, k_rb, k_rh, k_ch;
   int pair_heads;             // 1: tiles = two heads, same slots; 0: two slot tiles, one head
   int n_tiles;                // slot tiles of 128
   int items_per_kv;           // work items per (b, hk)
@@ -186,7 +193,9 @@ struct Cfg {
 // two blocks and the scores run two blocks ahead of the softmax; with 128 a block is the
 // whole K/V tile and the next scores of a tile follow its P V.
 template <int D, int KB>
-__global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_constant__ TcParams p) {
+__global__ void __launch_bounds__(kThreads, 1)
+fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtensorMap tm_q,
+              const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v) {
   extern __shared__ __align__(1024) uint8_t smem[];
   using C = Cfg<D>;
   constexpr int kHalf = KB;             // keys per score block
@@ -213,7 +222,7 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
     for (int i = 0; i < C::kNumBars; ++i)
       mbar_init(bar(i), (i >= C::kBarPReady && i < C::kBarPvDone) ? kTile
                         : (i == C::kBarQFull || (i >= C::kBarSlotFull && i < C::kBarSlotEmpty))
-                            ? kProducers : 1);
+                            ? (p.use_tma ? 1 : kProducers) : 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {
@@ -230,7 +239,77 @@ __global__ void __launch_bounds__(kThreads, 1) fwd_tc_kernel(const __grid_consta
   // whole score row each.
   if (warp < 4) {
   asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
-  if (warp >= 1) {
+  if (warp >= 1 && p.use_tma) {
+    // ------------------------------------------- tile loads by TMA (one thread of warp 1)
+    // Rows are consecutive tokens here, so a tile is D / 64 boxes of 128 rows x 64 columns
+    // that the TMA unit lays out in the same swizzled form the gather produces; no producer
+    // instructions compete with the softmax warps.  Rows past the sequence read the next
+    // rows of the matrix (or zeros past its end); the window mask never lets them count and
+    // their outputs are not stored.  The key-token lists are not written: the one-sided
+    // rule tests slots only.
+    if (threadIdx.x == 32) {
+      uint32_t use = 0, gt = 0, it = 0, q_armed = 0xffffffffu;
+      bool live = true;
+      auto load_tile = [&](const CUtensorMap* tm, uint32_t dst, int col, int64_t row, uint32_t mb) {
+#pragma unroll
+        for (int c = 0; c < D / 64; ++c)
+          tma_load_2d(dst + c * C::kChunkBytes, tm, col + 64 * c, (int)row, mb);
+      };
+      for (int w_item = blockIdx.x; w_item < p.total_items && live; w_item += gridDim.x, ++it) {
+        const int item = w_item % p.items_per_kv, bh = w_item / p.items_per_kv;
+        const int hk = bh % p.Hkv, b = bh / p.Hkv;
+        const Geo g = make_geo(p, item, hk);
+        const int64_t krow = b * p.k_rb + hk * p.k_rh + g.kstart;
+        const int kcol = (int)(hk * p.k_ch);
+        for (int j = 0; j < g.T; ++j, ++gt) {
+          if (use >= (uint32_t)C::kSlots)
+            live = mbar_wait(bar(C::kBarSlotEmpty + use % C::kSlots), (use / C::kSlots - 1) & 1u,
+                             gave_up, p.status);
+          if (!live) break;
+          mbar_arrive(bar(C::kBarTokFull + gt % C::kTok));
+          uint32_t mb = bar(C::kBarSlotFull + use % C::kSlots);
+          mbar_expect_tx(mb, C::kTileBytes);
+          load_tile(&tm_k, sbase + C::kOffRing + (use % C::kSlots) * C::kTileBytes, kcol,
+                    krow + j * kTile, mb);
+          ++use;
+          if (j == 0) {
+            if (it) live = mbar_wait(bar(C::kBarQEmpty), (it - 1) & 1u, gave_up, p.status);
+            if (!live) break;
+            mbar_expect_tx(bar(C::kBarQFull), 2 * C::kTileBytes);
+            q_armed = it;
+#pragma unroll
+            for (int t = 0; t < 2; ++t)
+              load_tile(&tm_q, sbase + C::kOffQ + t * C::kTileBytes, (int)(g.hq[t] * p.q_ch),
+                        b * p.q_rb + g.hq[t] * p.q_rh + g.q0[t], bar(C::kBarQFull));
+          }
+          if (use >= (uint32_t)C::kSlots)
+            live = mbar_wait(bar(C::kBarSlotEmpty + use % C::kSlots), (use / C::kSlots - 1) & 1u,
+                             gave_up, p.status);
+          if (!live) break;
+          mb = bar(C::kBarSlotFull + use % C::kSlots);
+          mbar_expect_tx(mb, C::kTileBytes);
+          load_tile(&tm_v, sbase + C::kOffRing + (use % C::kSlots) * C::kTileBytes, kcol,
+                    krow + j * kTile, mb);
+          ++use;
+        }
+      }
+      // loads that were started but never consumed (only after a failed wait) must land
+      // before the shared memory goes away: wait for them, again with a limit
+      if (!live || *gave_up) {
+        const uint32_t first = use > (uint32_t)C::kSlots ? use - C::kSlots : 0u;
+        for (uint32_t u = first; u < use; ++u)
+          for (int tries = 0; tries < 100000; ++tries) {
+            if (mbar_try(bar(C::kBarSlotFull + u % C::kSlots), (u / C::kSlots) & 1u)) break;
+            __nanosleep(100);
+          }
+        if (q_armed != 0xffffffffu)
+          for (int tries = 0; tries < 100000; ++tries) {
+            if (mbar_try(bar(C::kBarQFull), q_armed & 1u)) break;
+            __nanosleep(100);
+          }
+      }
+    }
+  } else if (warp >= 1) {
     // ---------------------------------------------------- gather producers (warps 1-3)
     // Each 16-byte piece of a row goes from global memory to its swizzled place in shared
     // memory with cp.async; one warp instruction moves kRpi whole rows.
@@ -743,6 +822,38 @@ bool key_block_128(int w) {
   return forced ? forced == 128 : w > 128;
 }
 
+// SA_SWA_TMA=0 keeps the cp.async gather for the one-sided SWA branch too (tests run both).
+bool swa_tma_disabled() {
+  static int v = -1;
+  if (v < 0) {
+    const char* e = getenv("SA_SWA_TMA");
+    v = (e && e[0] == '0') ? 1 : 0;
+  }
+  return v == 1;
+}
+
+// Row (b, h, token) of a tensor with element strides s[0..2] as row b * rb + h * rh + token
+// and first column h * ch of one 2-D matrix with pitch s[2]; false when the layout is not of
+// that kind.  Also gives the matrix extent.
+bool row_view(const int64_t s[3], int B, int H, int n, int d, int64_t* rb, int64_t* rh,
+              int64_t* ch, int64_t* rows, int64_t* cols) {
+  const int64_t ts = s[2];
+  if (ts < d || s[0] % ts != 0) return false;
+  *rb = s[0] / ts;
+  if (s[1] % ts == 0) {
+    *rh = s[1] / ts;
+    *ch = 0;
+    *cols = d;
+  } else {
+    if (s[1] * (H - 1) + d > ts) return false;
+    *rh = 0;
+    *ch = s[1];
+    *cols = s[1] * (H - 1) + d;
+  }
+  *rows = (B - 1) * *rb + (H - 1) * *rh + n;
+  return *rows < (1ll << 31) - 4 * kTile;
+}
+
 bool tc_disabled() {
   static int v = -1;
   if (v < 0) {
@@ -792,10 +903,22 @@ cudaError_t launch_fwd_tc(const FwdArgs& a, cudaStream_t st) {
   }
   const unsigned grid = (unsigned)min(p.total_items, sm_count[dev]);
   const bool wide = key_block_128(a.w);
+  // whole-tile TMA loads for the one-sided SWA branch when q and k/v are plain row matrices
+  CUtensorMap tm_q{}, tm_k{}, tm_v{};
+  if (a.swa && mg.one_sided && !swa_tma_disabled()) {
+    int64_t qrows, qcols, krows, kcols;
+    if (row_view(a.qs, a.B, a.Hq, a.n, a.d, &p.q_rb, &p.q_rh, &p.q_ch, &qrows, &qcols) &&
+        row_view(a.ks, a.B, a.Hkv, a.n, a.d, &p.k_rb, &p.k_rh, &p.k_ch, &krows, &kcols) &&
+        aligned16(a.q) && aligned16(a.k) && aligned16(a.v) &&
+        make_map(&tm_q, a.q, qrows, qcols, a.qs[2], kTile) &&
+        make_map(&tm_k, a.k, krows, kcols, a.ks[2], kTile) &&
+        make_map(&tm_v, a.v, krows, kcols, a.ks[2], kTile))
+      p.use_tma = 1;
+  }
   auto go = [&](auto kernel, int smem) {
     cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (err != cudaSuccess) return err;
-    kernel<<<grid, kThreads, smem, st>>>(p);
+    kernel<<<grid, kThreads, smem, st>>>(p, tm_q, tm_k, tm_v);
     return cudaSuccess;
   };
   if (a.d == 128)

@@ -126,6 +126,36 @@ def test_both_score_block_widths(block):
     assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
 
 
+def test_swa_branch_without_tma_tile_loads():
+    # the one-sided SWA branch loads whole tiles by TMA when its tensors are plain row
+    # matrices; a child process with SA_SWA_TMA=0 runs the cp.async gather on the same cases
+    import os, subprocess, sys
+    env = dict(os.environ, SA_SWA_TMA="0")
+    r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-m", "gpu", __file__, "-k",
+                        "test_swa_forward_small or test_gated_forward_small or "
+                        "test_gated_forward_both_combine_paths"],
+                       env=env, capture_output=True, text=True)
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+
+
+def test_swa_tma_path_ragged_tail_and_strides():
+    """One-sided SWA on the tensor-core path with n not a multiple of 128 (the last tile reads
+    rows of the next head, or past the matrix), several heads and batches, both layouts."""
+    B, Hq, Hkv, n, w = 2, 4, 2, 389, 200
+    flags = CAUSAL | SWA_ONE_SIDED
+    for d in (64, 128):
+        q, k, v = draw((B, Hq, n, d), (B, Hkv, n, d), torch.bfloat16, seed=40 + d)
+        ry, _ = oracle.swa_forward(as_f64(q), as_f64(k), as_f64(v), w, flags)
+        for token_major in (False, True):
+            if token_major:
+                dev = [t.permute(0, 2, 1, 3).contiguous().cuda().permute(0, 2, 1, 3) for t in (q, k, v)]
+            else:
+                dev = [t.cuda() for t in (q, k, v)]
+            y = sa.sa_swa_forward(dev[0], dev[1], dev[2], w, flags, y=torch.empty_like(dev[0]))
+            close(y, ry, torch.bfloat16, "d=%d token_major=%s" % (d, token_major))
+    assert sa.sa_read_status() == 0
+
+
 def test_identity_permutation_equals_swa_on_device():
     B, Hq, Hkv, n, d, w = 1, 2, 1, 333, 64, 17
     q, k, v = draw((B, Hq, n, d), (B, Hkv, n, d), torch.float32, seed=1)
