@@ -192,7 +192,8 @@ struct Cfg {
 // D: head dimension.  KB: keys per score block, 64 or 128.  With 64 a tile's S columns hold
 // two blocks and the scores run two blocks ahead of the softmax; with 128 a block is the
 // whole K/V tile and the next scores of a tile follow its P V.
-template <int D, int KB>
+// TMA: the instantiation for launches whose tiles come by TMA (p.use_tma).
+template <int D, int KB, bool TMA>
 __global__ void __launch_bounds__(kThreads, 1)
 fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtensorMap tm_q,
               const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v) {
@@ -238,8 +239,12 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
   // Registers move from the producer / issuer warps to the softmax warps, which hold a
   // whole score row each.
   if (warp < 4) {
-  asm volatile("setmaxnreg.dec.sync.aligned.u32 80;");
-  if (warp >= 1 && p.use_tma) {
+  // Registers per lane over the 12 warps: 4 x 56 + 8 x 224 = 2016, all that the launch holds
+  // (12 x 168).  The four warps of a warpgroup must ask for the same count, so the issuing
+  // warp and the producer warps go down together.  With 224 registers the 128 scores and the
+  // 32 packed probabilities of a softmax thread stay in registers (at 208 they spilled).
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+  if (warp >= 1 && TMA) {
     // ------------------------------------------- tile loads by TMA (one thread of warp 1)
     // Rows are consecutive tokens here, so a tile is D / 64 boxes of 128 rows x 64 columns
     // that the TMA unit lays out in the same swizzled form the gather produces; no producer
@@ -309,7 +314,7 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
           }
       }
     }
-  } else if (warp >= 1) {
+  } else if (warp >= 1 && !TMA) {
     // ---------------------------------------------------- gather producers (warps 1-3)
     // Each 16-byte piece of a row goes from global memory to its swizzled place in shared
     // memory with cp.async; one warp instruction moves kRpi whole rows.
@@ -560,7 +565,7 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
     __syncwarp();
   }
   } else {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 208;");
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
     // ------------------------------------------------- softmax and epilogue
     const int t = (warp - 4) / 4;
     const int row = threadIdx.x - 128 - t * 128;       // 0..127 == TMEM lane
@@ -921,10 +926,17 @@ cudaError_t launch_fwd_tc(const FwdArgs& a, cudaStream_t st) {
     kernel<<<grid, kThreads, smem, st>>>(p, tm_q, tm_k, tm_v);
     return cudaSuccess;
   };
+  const bool tma = p.use_tma != 0;
   if (a.d == 128)
-    e = wide ? go(fwd_tc_kernel<128, 128>, Cfg<128>::kBytes) : go(fwd_tc_kernel<128, 64>, Cfg<128>::kBytes);
+    e = wide ? (tma ? go(fwd_tc_kernel<128, 128, true>, Cfg<128>::kBytes)
+                    : go(fwd_tc_kernel<128, 128, false>, Cfg<128>::kBytes))
+             : (tma ? go(fwd_tc_kernel<128, 64, true>, Cfg<128>::kBytes)
+                    : go(fwd_tc_kernel<128, 64, false>, Cfg<128>::kBytes));
   else
-    e = wide ? go(fwd_tc_kernel<64, 128>, Cfg<64>::kBytes) : go(fwd_tc_kernel<64, 64>, Cfg<64>::kBytes);
+    e = wide ? (tma ? go(fwd_tc_kernel<64, 128, true>, Cfg<64>::kBytes)
+                    : go(fwd_tc_kernel<64, 128, false>, Cfg<64>::kBytes))
+             : (tma ? go(fwd_tc_kernel<64, 64, true>, Cfg<64>::kBytes)
+                    : go(fwd_tc_kernel<64, 64, false>, Cfg<64>::kBytes));
   if (e != cudaSuccess) return e;
   bump_launches();
   return cudaGetLastError();
