@@ -340,7 +340,7 @@ def extras(args, c, wl, sa, torch, dev, host, perm, inv, ws, y, pk):
     e2e_ms = event_ms(e2e_step, it, 2, torch)
     res["e2e"] = {"value": c.B * c.n / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms,
                   "h2d_bytes_per_step": hf.h2d_bytes(), "d2h_bytes_per_step": hf.d2h_bytes(),
-                  "api": "host.HostForward.forward, 8 KV-head groups on 3 streams"}
+                  "api": "host.HostForward.forward, 8 KV-head groups x 2 query-head parts on 3 streams"}
     del hf
 
     # backward on the pre-training shape (fresh permutation, gated forward saving, backward)

@@ -19,6 +19,17 @@ def test_head_groups_cover_every_head_once():
         assert kv_seen == list(range(Hkv)) and q_seen == list(range(Hq))
 
 
+def test_split_query_heads_keeps_coverage_and_kv_ownership():
+    g = host.split_query_heads(host.head_groups(32, 8, 8), 2)
+    assert len(g) == 16
+    assert [x[2:4] for x in g] == [(2 * i, 2 * i + 2) for i in range(16)]
+    assert [x[4] for x in g] == [True, False] * 8          # K/V travel with the first part only
+    assert all(kb - ka == 1 for ka, kb, *_ in g)
+    # ranges with several KV heads, or an odd number of query heads per KV head, stay whole
+    assert host.split_query_heads(host.head_groups(8, 4, 2), 2) == [(0, 2, 0, 4, True), (2, 4, 4, 8, True)]
+    assert host.split_query_heads(host.head_groups(3, 1, 1), 2) == [(0, 1, 0, 3, True)]
+
+
 def test_head_groups_rejects_bad_head_counts():
     with pytest.raises(ValueError):
         host.head_groups(10, 4, 2)
@@ -27,8 +38,8 @@ def test_head_groups_rejects_bad_head_counts():
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("n_groups", [1, 3, 4])
-def test_pipelined_forward_equals_single_call(n_groups):
+@pytest.mark.parametrize("n_groups,q_parts", [(1, 1), (3, 2), (4, 2), (4, 1)])
+def test_pipelined_forward_equals_single_call(n_groups, q_parts):
     from paper_2604_00754_b200 import binding as sa
     B, Hq, Hkv, n, d, w = 2, 8, 4, 1000, 64, 256
     g = torch.Generator().manual_seed(11)
@@ -37,7 +48,7 @@ def test_pipelined_forward_equals_single_call(n_groups):
     v = torch.randn(B, Hkv, n, d, generator=g).bfloat16().pin_memory()
     lg = torch.randn(2, Hq, generator=g).pin_memory()
     hy = torch.empty_like(q).pin_memory()
-    hf = host.HostForward(B, Hq, Hkv, n, d, w, n_groups=n_groups)
+    hf = host.HostForward(B, Hq, Hkv, n, d, w, n_groups=n_groups, q_parts=q_parts)
     hf.forward(q, k, v, lg, hy, seed=5, layer=2)
     torch.cuda.synchronize()
     perm, inv = sa.sa_make_perm(5, 2, B, n)
