@@ -15,7 +15,7 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
                : "memory");
 }
 // One box of the tensor map (x: element column, a multiple of 64; y: row) into shared memory;
-// the bytes are counted on the mbarrier.  No multicast.
+// the bytes are counted on the mbarrier.  A load into this CTA only.
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* tm, int x, int y,
                                             uint32_t bar) {
   asm volatile(
