@@ -160,3 +160,26 @@ def test_backward_model_width_single_path():
     assert sa.sa_read_status() == 0
     want = oracle.gate_projection_backward(dout.double().numpy(), ya.double().numpy(), wa.double().numpy())
     _check_grads(got, want, 2e-2)
+
+
+@pytest.mark.parametrize("rows,dm", [(1, 64), (127, 64), (130, 448)])
+def test_gate_edge_shapes_forward_and_backward(rows, dm):
+    """A single row, one row short of a tile, a ragged last row tile with a half column tile."""
+    from paper_2604_00754_b200 import binding as sa
+    ya, yb, wa, wb = _draw(rows, dm, 100 + rows, torch.bfloat16)
+    dout = torch.randn(rows, dm, generator=torch.Generator().manual_seed(rows)).bfloat16()
+    out = sa.sa_gate_projection_forward(ya.cuda(), wa.cuda(), yb.cuda(), wb.cuda())
+    got = sa.sa_gate_projection_backward(dout.cuda(), ya.cuda(), wa.cuda(), yb.cuda(), wb.cuda())
+    assert sa.sa_read_status() == 0
+    _check(out, ya, wa, yb, wb, dm, 2e-2)
+    want = oracle.gate_projection_backward(dout.double().numpy(), ya.double().numpy(), wa.double().numpy(),
+                                           yb.double().numpy(), wb.double().numpy())
+    _check_grads(got, want, 2e-2)
+
+
+def test_gate_backward_rejects_small_workspace():
+    from paper_2604_00754_b200 import binding as sa
+    y = torch.zeros(4, 64, dtype=torch.bfloat16, device="cuda")
+    w = torch.zeros(64, 64, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(sa.SaError):
+        sa.sa_gate_projection_backward(y, y, w, ws=torch.empty(16, dtype=torch.uint8, device="cuda"))
