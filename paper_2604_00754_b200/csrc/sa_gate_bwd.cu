@@ -1,8 +1,8 @@
 // Backward of the projection gates (Eq. 5-6): with z = y w^T, g = sigmoid(z), out = g * y,
 //   dz = dout * y * g * (1 - g),   dw = dz^T y,   dy = dout * g + dz w      (per path).
 // Three contractions per path, all on the 5th-generation tensor cores through one kernel
-// template (128 x 128 output tiles, TMA ring, double-buffered fp32 accumulators in tensor
-// memory, eight epilogue warps):
+// template (128 x 256 output tiles, or 128 x 128 for small products, TMA ring,
+// double-buffered fp32 accumulators in tensor memory, eight epilogue warps):
 //   kDz: z = y w^T        (both operands K-major);  epilogue writes dz and dout * g
 //   kDy: dz w             (w read with its rows as the contraction index: N-major operand);
 //                          epilogue adds dout * g and writes dy
@@ -19,14 +19,24 @@ namespace {
 
 enum BwdMode { kDz = 0, kDy = 1, kDw = 2 };
 
-constexpr int kT = 128, kBK = 64;
-constexpr int kStages = 3;
-constexpr int kTileBytes = kT * kBK * 2;          // one operand tile of one K chunk, either major
-constexpr int kStageBytes = 4 * kTileBytes;       // A, B of two consecutive K chunks
+constexpr int kT = 128, kBK = 64;                  // output tiles of 128 rows, K chunks of 64
+constexpr int kATileBytes = kT * kBK * 2;          // A of one K chunk, either major: 16 KB
+constexpr int kChunk = 64 * kBK * 2;               // 64 rows x 64 columns: one box of a row-contracted operand
+constexpr int kRingBytes = 12 * kATileBytes;       // 192 KB of operand stages
+// TN: columns of the output tile.  256 halves the operand bytes per flop of the B side and is
+// used when it still leaves at least one tile per SM; 128 otherwise.  A stage holds 64 KB or
+// 48 KB (two K chunks of A + B at TN = 128, one at TN = 256): eight or four products.
+template <int TN> struct Tile {
+  static constexpr int kCps = TN == 128 ? 2 : 1;                 // K chunks per stage
+  static constexpr int kBTileBytes = TN * kBK * 2;
+  static constexpr int kStageBytes = kCps * (kATileBytes + kBTileBytes);
+  static constexpr int kStages = kRingBytes / kStageBytes;       // 3 or 4
+};
+constexpr int kMaxStages = 4;
 constexpr int kThreadsB = 320;
-constexpr int kOffBars = kStages * kStageBytes;
-constexpr int kBarFull = 0, kBarEmpty = kStages, kBarAccFull = 2 * kStages,
-              kBarAccEmpty = 2 * kStages + 2, kNumBars = 2 * kStages + 4;
+constexpr int kOffBars = kRingBytes;
+constexpr int kBarFull = 0, kBarEmpty = kMaxStages, kBarAccFull = 2 * kMaxStages,
+              kBarAccEmpty = 2 * kMaxStages + 2, kNumBars = 2 * kMaxStages + 4;
 constexpr int kOffMisc = kOffBars + kNumBars * 8;
 constexpr int kSmemB = kOffMisc + 16;
 
@@ -37,7 +47,7 @@ struct BwdGateParams {
   __nv_bfloat16* out;              // kDy: dy, kDw: dw
   int64_t ld_y, ld_ws, ld_out;
   int64_t m_rows, n_cols;          // extent of the product
-  int tiles_m, tiles_n, k_pairs;   // k_pairs: hand-overs per tile (two K chunks each)
+  int tiles_m, tiles_n, k_pairs;   // k_pairs: hand-overs per tile (one or two K chunks each)
   int* status;
 };
 
@@ -50,14 +60,17 @@ __device__ __forceinline__ void mma_ss(uint32_t d, uint64_t a, uint64_t b, uint3
       : "memory");
 }
 // bit 15: A is MN-major, bit 16: B is MN-major
-__host__ __device__ constexpr uint32_t idesc_of(bool a_mn, bool b_mn) {
-  return instr_desc(kT, kT, b_mn) | ((a_mn ? 1u : 0u) << 15);
+__host__ __device__ constexpr uint32_t idesc_of(int tn, bool a_mn, bool b_mn) {
+  return instr_desc(kT, tn, b_mn) | ((a_mn ? 1u : 0u) << 15);
 }
-template <int MODE>
+template <int MODE, int TN>
 __global__ void __launch_bounds__(kThreadsB, 1)
 gate_bwd_kernel(const __grid_constant__ BwdGateParams p, const __grid_constant__ CUtensorMap tm_a,
                 const __grid_constant__ CUtensorMap tm_b) {
   constexpr bool kAmn = MODE == kDw, kBmn = MODE != kDz;
+  using TL = Tile<TN>;
+  constexpr int kStages = TL::kStages, kStageBytes = TL::kStageBytes, kTN = TN;
+  constexpr int kBlock = 2048 / TN;       // column tiles per block of the tile order
   extern __shared__ __align__(1024) uint8_t smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (*(volatile int*)p.status == SA_ERR_TIMEOUT) return;
@@ -77,7 +90,7 @@ gate_bwd_kernel(const __grid_constant__ BwdGateParams p, const __grid_constant__
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                 ::"r"(smem_u32(tmem_slot)), "r"(256u) : "memory");
+                 ::"r"(smem_u32(tmem_slot)), "r"(512u) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
@@ -85,13 +98,13 @@ gate_bwd_kernel(const __grid_constant__ BwdGateParams p, const __grid_constant__
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   const int total = p.tiles_m * p.tiles_n;
-  // blocks of 16 column tiles, row tile by row tile inside a block (operand slices stay in L2)
+  // blocks of 2048 columns, row tile by row tile inside a block (operand slices stay in L2)
   auto origin = [&](int tile, int* m0, int* n0) {
-    const int per_block = p.tiles_m * 16;
+    const int per_block = p.tiles_m * kBlock;
     const int nb = tile / per_block, rem = tile - nb * per_block;
-    const int width = min(16, p.tiles_n - nb * 16);
+    const int width = min(kBlock, p.tiles_n - nb * kBlock);
     *m0 = (rem / width) * kT;
-    *n0 = (nb * 16 + rem % width) * kT;
+    *n0 = (nb * kBlock + rem % width) * kTN;
   };
 
   if (warp == 0) {
@@ -110,18 +123,18 @@ gate_bwd_kernel(const __grid_constant__ BwdGateParams p, const __grid_constant__
           const uint32_t dst = sbase + s * kStageBytes, fb = bar(kBarFull + s);
           mbar_expect_tx(fb, kStageBytes);
 #pragma unroll
-          for (int c = 0; c < 2; ++c) {
-            const int k0 = (2 * kp + c) * kBK;       // past the end: zeros
-            const uint32_t da = dst + (2 * c) * kTileBytes, db = da + kTileBytes;
+          for (int q = 0; q < TL::kCps; ++q) {
+            const int k0 = (TL::kCps * kp + q) * kBK;                   // past the end: zeros
+            const uint32_t da = dst + q * (kATileBytes + TL::kBTileBytes), db = da + kATileBytes;
             if (kAmn) {
-              tma_load_2d(da, &tm_a, m0, k0, fb);
-              tma_load_2d(da + kTileBytes / 2, &tm_a, m0 + 64, k0, fb);
+#pragma unroll
+              for (int c = 0; c < kT / 64; ++c) tma_load_2d(da + c * kChunk, &tm_a, m0 + 64 * c, k0, fb);
             } else {
               tma_load_2d(da, &tm_a, k0, m0, fb);
             }
             if (kBmn) {
-              tma_load_2d(db, &tm_b, n0, k0, fb);
-              tma_load_2d(db + kTileBytes / 2, &tm_b, n0 + 64, k0, fb);
+#pragma unroll
+              for (int c = 0; c < kTN / 64; ++c) tma_load_2d(db + c * kChunk, &tm_b, n0 + 64 * c, k0, fb);
             } else {
               tma_load_2d(db, &tm_b, k0, n0, fb);
             }
@@ -141,10 +154,10 @@ gate_bwd_kernel(const __grid_constant__ BwdGateParams p, const __grid_constant__
   } else if (warp == 1) {
     // -------------------------------------------------------------------- MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = idesc_of(kAmn, kBmn);
+      constexpr uint32_t idesc = idesc_of(TN, kAmn, kBmn);
       constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
       constexpr uint32_t kLoK = (16u >> 4) << 16;                       // K-major operand
-      constexpr uint32_t kLoMN = ((uint32_t)(kTileBytes / 2) >> 4) << 16;  // next 64 columns
+      constexpr uint32_t kLoMN = ((uint32_t)kChunk >> 4) << 16;           // next 64 columns
       constexpr uint32_t kStepK = 32u >> 4, kStepMN = 2048u >> 4;         // one K step of 16
       uint32_t use = 0, it = 0;
       bool ok = true;
@@ -154,7 +167,7 @@ gate_bwd_kernel(const __grid_constant__ BwdGateParams p, const __grid_constant__
           ok = mbar_wait(bar(kBarAccEmpty + buf), (it / 2 - 1) & 1u, gave_up, p.status);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t d = tmem + buf * 128;
+        const uint32_t d = tmem + buf * kTN;
         for (int kp = 0; kp < p.k_pairs && ok; ++kp, ++use) {
           const uint32_t s = use % kStages;
           ok = mbar_wait(bar(kBarFull + s), (use / kStages) & 1u, gave_up, p.status);
@@ -162,13 +175,14 @@ gate_bwd_kernel(const __grid_constant__ BwdGateParams p, const __grid_constant__
           tc_fence_after();
           const uint32_t lo = (sbase + s * kStageBytes) >> 4;
 #pragma unroll
-          for (int c = 0; c < 2; ++c) {
-            const uint64_t a0 = desc64((lo + (2 * c) * (kTileBytes >> 4)) | (kAmn ? kLoMN : kLoK), kDescHi);
-            const uint64_t b0 = desc64((lo + (2 * c + 1) * (kTileBytes >> 4)) | (kBmn ? kLoMN : kLoK), kDescHi);
+          for (int q = 0; q < TL::kCps; ++q) {
+            const uint32_t la = lo + q * ((kATileBytes + TL::kBTileBytes) >> 4);
+            const uint64_t a0 = desc64(la | (kAmn ? kLoMN : kLoK), kDescHi);
+            const uint64_t b0 = desc64((la + (kATileBytes >> 4)) | (kBmn ? kLoMN : kLoK), kDescHi);
 #pragma unroll
             for (int ks = 0; ks < 4; ++ks)
               mma_ss(d, a0 + ks * (kAmn ? kStepMN : kStepK), b0 + ks * (kBmn ? kStepMN : kStepK),
-                     idesc, (kp > 0 || c > 0 || ks > 0) ? 1u : 0u);
+                     idesc, (kp > 0 || q > 0 || ks > 0) ? 1u : 0u);
           }
           tc_commit(bar(kBarEmpty + s));
         }
@@ -194,9 +208,9 @@ gate_bwd_kernel(const __grid_constant__ BwdGateParams p, const __grid_constant__
       const int64_t r = (int64_t)m0 + row;
       const bool row_ok = r < p.m_rows;
 #pragma unroll 1
-      for (int c = 2 * half; c < 2 * half + 2; ++c) {
+      for (int c = (kTN / 64) * half; c < (kTN / 64) * (half + 1); ++c) {
         uint32_t acc[32];
-        tmem_ld32(tmem + lane_addr + buf * 128 + 32 * c, acc);
+        tmem_ld32(tmem + lane_addr + buf * kTN + 32 * c, acc);
         tmem_wait_ld();
         const int col = n0 + 32 * c;
         if (row_ok && col < p.n_cols) {
@@ -251,7 +265,7 @@ gate_bwd_kernel(const __grid_constant__ BwdGateParams p, const __grid_constant__
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(256u)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u)
                  : "memory");
   }
 }
@@ -301,18 +315,24 @@ __global__ void dw_simt_kernel(int64_t rows, int dm, const float* __restrict__ d
 
 // ------------------------------------------------------------------------------ host
 
-template <int MODE>
+// Wide (128 x 256) tiles when they still give every SM at least two tiles.
+bool wide_tiles(int64_t m_rows, int64_t n_cols, int sms) {
+  return ((m_rows + kT - 1) / kT) * ((n_cols + 255) / 256) >= 2 * (int64_t)sms;
+}
+
+template <int MODE, int TN>
 cudaError_t launch_mode(BwdGateParams p, const CUtensorMap& a, const CUtensorMap& b, int64_t k,
                         int sms, cudaStream_t st) {
   p.tiles_m = (int)((p.m_rows + kT - 1) / kT);
-  p.tiles_n = (int)((p.n_cols + kT - 1) / kT);
-  p.k_pairs = (int)((k + 2 * kBK - 1) / (2 * kBK));
-  cudaError_t e = cudaFuncSetAttribute(gate_bwd_kernel<MODE>,
+  p.tiles_n = (int)((p.n_cols + TN - 1) / TN);
+  const int per = Tile<TN>::kCps * kBK;
+  p.k_pairs = (int)((k + per - 1) / per);
+  cudaError_t e = cudaFuncSetAttribute(gate_bwd_kernel<MODE, TN>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemB);
   if (e != cudaSuccess) return e;
   const int64_t total = (int64_t)p.tiles_m * p.tiles_n;
   const unsigned grid = (unsigned)(total < sms ? total : sms);
-  gate_bwd_kernel<MODE><<<grid, kThreadsB, kSmemB, st>>>(p, a, b);
+  gate_bwd_kernel<MODE, TN><<<grid, kThreadsB, kSmemB, st>>>(p, a, b);
   bump_launches();
   return cudaGetLastError();
 }
@@ -362,8 +382,10 @@ extern "C" sa_status sa_gate_projection_backward(
     if (tc) {
       __nv_bfloat16* dz = (__nv_bfloat16*)ws;
       __nv_bfloat16* dyd = dz + rows * (int64_t)dm;
+      const bool wide_r = wide_tiles(rows, dm, sms), wide_w = wide_tiles(dm, dm, sms);
       CUtensorMap y_k, w_k, dz_k, w_mn, dz_mn, y_mn;
-      if (!make_map(&y_k, y, rows, dm, ld_y, 128) || !make_map(&w_k, w, dm, dm, dm, 128) ||
+      if (!make_map(&y_k, y, rows, dm, ld_y, 128) ||
+          !make_map(&w_k, w, dm, dm, dm, wide_r ? 256 : 128) ||
           !make_map(&dz_k, dz, rows, dm, dm, 128) || !make_map(&w_mn, w, dm, dm, dm, 64) ||
           !make_map(&dz_mn, dz, rows, dm, dm, 64) || !make_map(&y_mn, y, rows, dm, ld_y, 64))
         return SA_ERR_CUDA;
@@ -373,14 +395,20 @@ extern "C" sa_status sa_gate_projection_backward(
       // z = y w^T; epilogue: dz, dout * g
       p.dout = (const __nv_bfloat16*)dout; p.y = (const __nv_bfloat16*)y; p.ld_out = ld_dout;
       p.m_rows = rows; p.n_cols = dm;
-      if (launch_mode<kDz>(p, y_k, w_k, dm, sms, st) != cudaSuccess) return SA_ERR_CUDA;
+      if ((wide_r ? launch_mode<kDz, 256>(p, y_k, w_k, dm, sms, st)
+                  : launch_mode<kDz, 128>(p, y_k, w_k, dm, sms, st)) != cudaSuccess)
+        return SA_ERR_CUDA;
       // dy = dz w + dout * g
       p.out = (__nv_bfloat16*)dy; p.ld_out = ld_dy;
-      if (launch_mode<kDy>(p, dz_k, w_mn, dm, sms, st) != cudaSuccess) return SA_ERR_CUDA;
+      if ((wide_r ? launch_mode<kDy, 256>(p, dz_k, w_mn, dm, sms, st)
+                  : launch_mode<kDy, 128>(p, dz_k, w_mn, dm, sms, st)) != cudaSuccess)
+        return SA_ERR_CUDA;
       // dw = dz^T y
       p.out = (__nv_bfloat16*)dw; p.ld_out = dm;
       p.m_rows = dm; p.n_cols = dm;
-      if (launch_mode<kDw>(p, dz_mn, y_mn, rows, sms, st) != cudaSuccess) return SA_ERR_CUDA;
+      if ((wide_w ? launch_mode<kDw, 256>(p, dz_mn, y_mn, rows, sms, st)
+                  : launch_mode<kDw, 128>(p, dz_mn, y_mn, rows, sms, st)) != cudaSuccess)
+        return SA_ERR_CUDA;
     } else {
       float* dz = (float*)ws;
       float* dyd = dz + rows * (int64_t)dm;
