@@ -158,6 +158,10 @@ cudaError_t launch_combine(void* y, const void* y_sa, const void* y_swa, const f
                            int B, int Hq, int n, int d, const int64_t s[3], int dtype,
                            cudaStream_t st);
 
+bool gate_forward_wide(int64_t rows, int dm, const void* y_sa, const void* y_swa, int64_t ld_y,
+                       const void* w_sa, const void* w_swa, void* out, int64_t ld_out,
+                       int* status, int sms, cudaStream_t st, cudaError_t* err);
+
 cudaError_t launch_bwd_simt(const BwdArgs& a, int dtype, cudaStream_t st);
 size_t bwd_ws_bytes(int B, int Hq, int n, int* chunks_out);
 

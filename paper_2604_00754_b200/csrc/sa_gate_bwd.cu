@@ -17,7 +17,7 @@
 namespace sa {
 namespace {
 
-enum BwdMode { kDz = 0, kDy = 1, kDw = 2 };
+enum BwdMode { kDz = 0, kDy = 1, kDw = 2, kFwd = 3 };   // kFwd: the forward's sigmoid(y w^T) * y
 
 constexpr int kT = 128, kBK = 64;                  // output tiles of 128 rows, K chunks of 64
 constexpr int kATileBytes = kT * kBK * 2;          // A of one K chunk, either major: 16 KB
@@ -48,6 +48,7 @@ struct BwdGateParams {
   int64_t ld_y, ld_ws, ld_out;
   int64_t m_rows, n_cols;          // extent of the product
   int tiles_m, tiles_n, k_pairs;   // k_pairs: hand-overs per tile (one or two K chunks each)
+  int accum;                       // kFwd: add to what out already holds (second path)
   int* status;
 };
 
@@ -67,7 +68,7 @@ template <int MODE, int TN>
 __global__ void __launch_bounds__(kThreadsB, 1)
 gate_bwd_kernel(const __grid_constant__ BwdGateParams p, const __grid_constant__ CUtensorMap tm_a,
                 const __grid_constant__ CUtensorMap tm_b) {
-  constexpr bool kAmn = MODE == kDw, kBmn = MODE != kDz;
+  constexpr bool kAmn = MODE == kDw, kBmn = MODE == kDy || MODE == kDw;
   using TL = Tile<TN>;
   constexpr int kStages = TL::kStages, kStageBytes = TL::kStageBytes, kTN = TN;
   constexpr int kBlock = 2048 / TN;       // column tiles per block of the tile order
@@ -213,6 +214,20 @@ gate_bwd_kernel(const __grid_constant__ BwdGateParams p, const __grid_constant__
         tmem_ld32(tmem + lane_addr + buf * kTN + 32 * c, acc);
         tmem_wait_ld();
         const int col = n0 + 32 * c;
+        // the epilogue's row reads are requested together, ahead of the stores they may not
+        // pass (the outputs may alias the inputs as far as the compiler knows), so that their
+        // latencies overlap: fy = y (kDz, kFwd) or dout * g (kDy), fo = dout (kDz) or out (kFwd)
+        uint4 fy[4], fo[4];
+        if (MODE != kDw && row_ok && col < p.n_cols) {
+#pragma unroll
+          for (int x8 = 0; x8 < 4; ++x8) {
+            const int64_t e = col + 8 * x8;
+            if (MODE == kDy) fy[x8] = *reinterpret_cast<const uint4*>(p.dyd + r * p.ld_ws + e);
+            else fy[x8] = *reinterpret_cast<const uint4*>(p.y + r * p.ld_y + e);
+            if (MODE == kDz || (MODE == kFwd && p.accum))
+              fo[x8] = *reinterpret_cast<const uint4*>((MODE == kDz ? p.dout : p.out) + r * p.ld_out + e);
+          }
+        }
         if (row_ok && col < p.n_cols) {
 #pragma unroll
           for (int x8 = 0; x8 < 4; ++x8) {
@@ -223,10 +238,8 @@ gate_bwd_kernel(const __grid_constant__ BwdGateParams p, const __grid_constant__
             uint4 st;
             __nv_bfloat162* hs = reinterpret_cast<__nv_bfloat162*>(&st);
             if (MODE == kDz) {
-              const uint4 vy = *reinterpret_cast<const uint4*>(p.y + r * p.ld_y + e);
-              const uint4 vd = *reinterpret_cast<const uint4*>(p.dout + r * p.ld_out + e);
-              const __nv_bfloat162* hy = reinterpret_cast<const __nv_bfloat162*>(&vy);
-              const __nv_bfloat162* hd = reinterpret_cast<const __nv_bfloat162*>(&vd);
+              const __nv_bfloat162* hy = reinterpret_cast<const __nv_bfloat162*>(&fy[x8]);
+              const __nv_bfloat162* hd = reinterpret_cast<const __nv_bfloat162*>(&fo[x8]);
               uint4 st2;
               __nv_bfloat162* hs2 = reinterpret_cast<__nv_bfloat162*>(&st2);
 #pragma unroll
@@ -239,10 +252,28 @@ gate_bwd_kernel(const __grid_constant__ BwdGateParams p, const __grid_constant__
               }
               *reinterpret_cast<uint4*>(p.dz + r * p.ld_ws + e) = st;
               *reinterpret_cast<uint4*>(p.dyd + r * p.ld_ws + e) = st2;
+            } else if (MODE == kFwd) {
+              const __nv_bfloat162* hy = reinterpret_cast<const __nv_bfloat162*>(&fy[x8]);
+#pragma unroll
+              for (int x = 0; x < 4; ++x) {
+                v8[2 * x] = logistic(v8[2 * x]) * __low2float(hy[x]);
+                v8[2 * x + 1] = logistic(v8[2 * x + 1]) * __high2float(hy[x]);
+              }
+              uint4* dst = reinterpret_cast<uint4*>(p.out + r * p.ld_out + e);
+              if (p.accum) {
+                const __nv_bfloat162* ho = reinterpret_cast<const __nv_bfloat162*>(&fo[x8]);
+#pragma unroll
+                for (int x = 0; x < 4; ++x) {
+                  v8[2 * x] += __low2float(ho[x]);
+                  v8[2 * x + 1] += __high2float(ho[x]);
+                }
+              }
+#pragma unroll
+              for (int x = 0; x < 4; ++x) hs[x] = __floats2bfloat162_rn(v8[2 * x], v8[2 * x + 1]);
+              *dst = st;
             } else {
               if (MODE == kDy) {
-                const uint4 vp = *reinterpret_cast<const uint4*>(p.dyd + r * p.ld_ws + e);
-                const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&vp);
+                const __nv_bfloat162* hp = reinterpret_cast<const __nv_bfloat162*>(&fy[x8]);
 #pragma unroll
                 for (int x = 0; x < 4; ++x) {
                   v8[2 * x] += __low2float(hp[x]);
@@ -338,6 +369,35 @@ cudaError_t launch_mode(BwdGateParams p, const CUtensorMap& a, const CUtensorMap
 }
 
 }  // namespace
+
+// Forward of one or two paths with 128 x 256 tiles, one launch per path (the second adds to
+// the first's rounded result); false when the product is too small for wide tiles to fill
+// the GPU, and the caller's fused kernel should run instead.
+bool gate_forward_wide(int64_t rows, int dm, const void* y_sa, const void* y_swa, int64_t ld_y,
+                       const void* w_sa, const void* w_swa, void* out, int64_t ld_out,
+                       int* status, int sms, cudaStream_t st, cudaError_t* err) {
+  *err = cudaSuccess;
+  if (!wide_tiles(rows, dm, sms)) return false;
+  for (int x = 0; x < (y_swa ? 2 : 1); ++x) {
+    const void* y = x ? y_swa : y_sa;
+    const void* w = x ? w_swa : w_sa;
+    CUtensorMap y_k, w_k;
+    if (!make_map(&y_k, y, rows, dm, ld_y, 128) || !make_map(&w_k, w, dm, dm, dm, 256)) {
+      *err = cudaErrorUnknown;
+      return true;
+    }
+    BwdGateParams p{};
+    p.status = status;
+    p.y = (const __nv_bfloat16*)y; p.ld_y = ld_y;
+    p.out = (__nv_bfloat16*)out; p.ld_out = ld_out;
+    p.m_rows = rows; p.n_cols = dm;
+    p.accum = x;
+    *err = launch_mode<kFwd, 256>(p, y_k, w_k, dm, sms, st);
+    if (*err != cudaSuccess) return true;
+  }
+  return true;
+}
+
 }  // namespace sa
 
 extern "C" size_t sa_gate_projection_backward_ws_bytes(int64_t rows, int32_t dm) {

@@ -177,6 +177,16 @@ gate_tc_kernel(const __grid_constant__ GateParams p, const __grid_constant__ CUt
       __nv_bfloat16* o = p.out + r * p.ld_out + n0;
 #pragma unroll 1
       for (int c = 2 * half; c < 2 * half + 2; ++c) {
+        // the rows of Y are requested together, ahead of the stores they may not pass (out may
+        // alias them as far as the compiler knows), so that their latencies overlap
+        uint4 fa[4], fb[4];
+        if (row_ok && n0 + 32 * c < p.dm) {
+#pragma unroll
+          for (int x8 = 0; x8 < 4; ++x8) {
+            fa[x8] = *reinterpret_cast<const uint4*>(ya + 32 * c + 8 * x8);
+            if (p.dual) fb[x8] = *reinterpret_cast<const uint4*>(yb + 32 * c + 8 * x8);
+          }
+        }
         uint32_t za[32], zb[32];
         tmem_ld32(tmem + lane_addr + buf * 256 + 32 * c, za);
         if (p.dual) tmem_ld32(tmem + lane_addr + buf * 256 + 128 + 32 * c, zb);
@@ -184,8 +194,7 @@ gate_tc_kernel(const __grid_constant__ GateParams p, const __grid_constant__ CUt
         if (row_ok && n0 + 32 * c < p.dm) {       // dm is a multiple of 64: whole chunks only
 #pragma unroll
           for (int x8 = 0; x8 < 4; ++x8) {
-            const uint4 va = *reinterpret_cast<const uint4*>(ya + 32 * c + 8 * x8);
-            const __nv_bfloat162* ha = reinterpret_cast<const __nv_bfloat162*>(&va);
+            const __nv_bfloat162* ha = reinterpret_cast<const __nv_bfloat162*>(&fa[x8]);
             float r8[8];
 #pragma unroll
             for (int x = 0; x < 4; ++x) {
@@ -193,8 +202,7 @@ gate_tc_kernel(const __grid_constant__ GateParams p, const __grid_constant__ CUt
               r8[2 * x + 1] = logistic(__uint_as_float(za[8 * x8 + 2 * x + 1])) * __high2float(ha[x]);
             }
             if (p.dual) {
-              const uint4 vb = *reinterpret_cast<const uint4*>(yb + 32 * c + 8 * x8);
-              const __nv_bfloat162* hb = reinterpret_cast<const __nv_bfloat162*>(&vb);
+              const __nv_bfloat162* hb = reinterpret_cast<const __nv_bfloat162*>(&fb[x8]);
 #pragma unroll
               for (int x = 0; x < 4; ++x) {
                 r8[2 * x] = fmaf(logistic(__uint_as_float(zb[8 * x8 + 2 * x])), __low2float(hb[x]),
@@ -278,6 +286,25 @@ extern "C" sa_status sa_gate_projection_forward(int64_t rows, int32_t dm, int32_
                   aligned16(y_sa) && aligned16(w_sa) && aligned16(out) &&
                   (!y_swa || (aligned16(y_swa) && aligned16(w_swa))) &&
                   rows < (1ll << 31) - 128;
+  // Large products run one 128 x 256-tile launch per path (a quarter fewer operand bytes per
+  // flop; the second path adds to the rounded result of the first); the fused dual-accumulator
+  // kernel below serves the rest, and everything with SA_GATE_WIDE=0 (tests run both).
+  static int wide_on = -1;
+  if (wide_on < 0) {
+    const char* e = getenv("SA_GATE_WIDE");
+    wide_on = (e && e[0] == '0') ? 0 : 1;
+  }
+  if (tc && wide_on) {
+    int dev = 0, sms = 0;
+    int* status = status_ptr();
+    if (!status || cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+      return SA_ERR_CUDA;
+    cudaError_t err;
+    if (gate_forward_wide(rows, dm, y_sa, y_swa, ld_y, w_sa, w_swa, out, ld_out, status, sms, st,
+                          &err))
+      return err == cudaSuccess ? SA_OK : SA_ERR_CUDA;
+  }
   if (tc) {
     CUtensorMap tm[4];
     const void* ysw = y_swa ? y_swa : y_sa;      // unused maps still have to be valid
