@@ -29,6 +29,8 @@
 // Warp roles: warp 0 MMA issuer and TMEM allocator, warps 1-3 gather producers, then one
 // (NBUF = 1) or two (NBUF = 2) warpgroups with one thread per row.  Every mbarrier wait is
 // bounded.
+#include <type_traits>
+
 #include "sa_bwd_tc.cuh"
 #include "sa_tc_common.cuh"
 
@@ -329,10 +331,12 @@ bwd_tc_kernel(const __grid_constant__ BwdTcParams p) {
     const bool tok_rule = p.causal && !p.one_sided;     // token order decides, not slots
     // rows = queries: mask key tokens above the query's; rows = keys: query tokens below
     const int cmp = tok_rule ? rtok : (kKeys ? (int)0x80000000 : 0x7fffffff);
+    // exp2(s * scale2 - lse2 + log2(scale)) is P * scale at once: dS needs no further multiply
+    const float l2scale = __log2f(p.scale), inv_scale = 1.f / p.scale;
     float lse2_r = 0.f, delta_r = 0.f, g = 1.f;
     if (!kKeys) {
       const size_t o = ((size_t)b * p.Hq + hr) * p.n + rtok;
-      lse2_r = p.lse[o] * kLog2e;
+      lse2_r = p.lse[o] * kLog2e - l2scale;
       delta_r = p.delta[o];
       if (p.gate_logit) g = 1.f / (1.f + __expf(-p.gate_logit[hr]));
     }
@@ -362,20 +366,34 @@ bwd_tc_kernel(const __grid_constant__ BwdTcParams p) {
       ok = __all_sync(0xffffffffu, ok);   // the tensor-memory accesses below are warp-collective
       if (C::kRowWgs == 1 && !ok) break;
       if (ok) tc_fence_after();
-      // visible columns of this row: one interval [lo, lo + span], cut by the token order
+      // visible columns of a row at slot rs: one interval [lo, hi], cut by the token order
       const int cb = cstart + j * KC;
+      auto interval = [&](int rs, int* lo_out, int* hi_out) {
+        int lo, hi;
+        if (p.one_sided) {
+          if (kKeys) { lo = rs - cb; hi = p.full_range ? p.n - 1 - cb : rs + (p.w - 1) - cb; }
+          else { lo = p.full_range ? -cb : rs - (p.w - 1) - cb; hi = rs - cb; }
+        } else if (p.full_range && !p.linear) { lo = -cb; hi = p.n - 1 - cb; }
+        else { lo = rs - p.h - cb; hi = rs + p.h - cb; }
+        if (p.linear || p.full_range || p.one_sided) {
+          lo = max(lo, -cb);
+          hi = min(hi, p.n - 1 - cb);
+        }
+        if (hi < lo) { lo = 1 << 30; hi = lo; }
+        *lo_out = lo;
+        *hi_out = hi;
+      };
       int lo, hi;
-      if (p.one_sided) {
-        if (kKeys) { lo = rslot - cb; hi = p.full_range ? p.n - 1 - cb : rslot + (p.w - 1) - cb; }
-        else { lo = p.full_range ? -cb : rslot - (p.w - 1) - cb; hi = rslot - cb; }
-      } else if (p.full_range && !p.linear) { lo = -cb; hi = p.n - 1 - cb; }
-      else { lo = rslot - p.h - cb; hi = rslot + p.h - cb; }
-      if (p.linear || p.full_range || p.one_sided) {
-        lo = max(lo, -cb);
-        hi = min(hi, p.n - 1 - cb);
-      }
-      if (hi < lo) { lo = 1 << 30; hi = lo; }
+      interval(rslot, &lo, &hi);
       const uint32_t span = (uint32_t)(hi - lo);
+      // Every row of the tile sees every column of this tile (up to the token order) when the
+      // last row's interval starts at or before column 0 and the first row's ends at or after
+      // the last column: then the per-element interval test is left out.
+      int lo_last, hi_last, lo_first, hi_first;
+      interval(r0 + kTile - 1, &lo_last, &hi_last);
+      interval(r0, &lo_first, &hi_first);
+      const bool interior = lo_last <= 0 && hi_first >= KC - 1 && hi_last >= KC - 1 &&
+                            lo_first <= 0 && r0 + kTile - 1 < p.n;
       const int32_t* coltok = reinterpret_cast<const int32_t*>(smem + C::kOffColTok) + s * kTile;
       const float* colvec = reinterpret_cast<const float*>(smem + C::kOffColVec) + s * 2 * kTile;
 #pragma unroll 1
@@ -388,6 +406,8 @@ bwd_tc_kernel(const __grid_constant__ BwdTcParams p) {
         }
         if (C::kRowWgs == 2 && rows_sync_stop(!ok)) { ok = false; break; }
         uint32_t ds_pk[16], p_pk[16];
+        auto chunk = [&](auto inter_c) {
+        constexpr bool kInter = decltype(inter_c)::value;
 #pragma unroll
         for (int x = 0; x < 32; x += 4) {
           const int col = 32 * c + x;
@@ -396,20 +416,22 @@ bwd_tc_kernel(const __grid_constant__ BwdTcParams p) {
           float4 d4 = make_float4(delta_r, delta_r, delta_r, delta_r);
           if (kKeys) {
             l4 = *reinterpret_cast<const float4*>(colvec + col);
-            l4.x *= kLog2e; l4.y *= kLog2e; l4.z *= kLog2e; l4.w *= kLog2e;
+            l4.x = fmaf(l4.x, kLog2e, -l2scale); l4.y = fmaf(l4.y, kLog2e, -l2scale);
+            l4.z = fmaf(l4.z, kLog2e, -l2scale); l4.w = fmaf(l4.w, kLog2e, -l2scale);
             d4 = *reinterpret_cast<const float4*>(colvec + kTile + col);
           }
           const int ctk[4] = {ct.x, ct.y, ct.z, ct.w};
           const float lv[4] = {l4.x, l4.y, l4.z, l4.w}, dl[4] = {d4.x, d4.y, d4.z, d4.w};
           float pv[4], dsv[4];
+          const float gp = g * inv_scale;
 #pragma unroll
           for (int y = 0; y < 4; ++y) {
-            const bool vis = (uint32_t)(col + y - lo) <= span &&
+            const bool vis = (kInter || (uint32_t)(col + y - lo) <= span) &&
                              (kKeys ? ctk[y] >= cmp : ctk[y] <= cmp);
             const float e = exp2f(fmaf(__uint_as_float(sv[x + y]), p.scale2, -lv[y]));
-            pv[y] = vis ? e : 0.f;
-            dsv[y] = pv[y] * (g * __uint_as_float(dv[x + y]) - dl[y]) * p.scale;
-            pv[y] *= g;
+            const float ps = vis ? e : 0.f;                       // P * scale
+            dsv[y] = ps * fmaf(g, __uint_as_float(dv[x + y]), -dl[y]);
+            pv[y] = ps * gp;                                      // g P, for dV
           }
           const __nv_bfloat162 a0 = __floats2bfloat162_rn(dsv[0], dsv[1]);
           const __nv_bfloat162 a1 = __floats2bfloat162_rn(dsv[2], dsv[3]);
@@ -422,6 +444,9 @@ bwd_tc_kernel(const __grid_constant__ BwdTcParams p) {
             p_pk[x / 2 + 1] = *reinterpret_cast<const uint32_t*>(&b1);
           }
         }
+        };
+        if (interior) chunk(std::true_type{});
+        else chunk(std::false_type{});
         // bf16 results go back over the columns already consumed (16 c .. 16 c + 15)
         tmem_st16(trow + C::kColS + buf + 16 * c, ds_pk);
         if (kKeys) tmem_st16(trow + C::kColP + buf + 16 * c, p_pk);
