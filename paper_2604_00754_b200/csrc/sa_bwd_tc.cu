@@ -424,14 +424,24 @@ bwd_tc_kernel(const __grid_constant__ BwdTcParams p) {
           const float lv[4] = {l4.x, l4.y, l4.z, l4.w}, dl[4] = {d4.x, d4.y, d4.z, d4.w};
           float pv[4], dsv[4];
           const float gp = g * inv_scale;
+          // two elements per instruction where the operation has a packed form
+          const float2 sc2 = make_float2(p.scale2, p.scale2), g2 = make_float2(g, g);
 #pragma unroll
-          for (int y = 0; y < 4; ++y) {
-            const bool vis = (kInter || (uint32_t)(col + y - lo) <= span) &&
-                             (kKeys ? ctk[y] >= cmp : ctk[y] <= cmp);
-            const float e = exp2f(fmaf(__uint_as_float(sv[x + y]), p.scale2, -lv[y]));
-            const float ps = vis ? e : 0.f;                       // P * scale
-            dsv[y] = ps * fmaf(g, __uint_as_float(dv[x + y]), -dl[y]);
-            pv[y] = ps * gp;                                      // g P, for dV
+          for (int y = 0; y < 4; y += 2) {
+            const bool vis0 = (kInter || (uint32_t)(col + y - lo) <= span) &&
+                              (kKeys ? ctk[y] >= cmp : ctk[y] <= cmp);
+            const bool vis1 = (kInter || (uint32_t)(col + y + 1 - lo) <= span) &&
+                              (kKeys ? ctk[y + 1] >= cmp : ctk[y + 1] <= cmp);
+            const float2 a = __ffma2_rn(make_float2(__uint_as_float(sv[x + y]), __uint_as_float(sv[x + y + 1])),
+                                        sc2, make_float2(-lv[y], -lv[y + 1]));
+            const float2 ps = make_float2(vis0 ? exp2f(a.x) : 0.f, vis1 ? exp2f(a.y) : 0.f);   // P * scale
+            const float2 in = __ffma2_rn(g2, make_float2(__uint_as_float(dv[x + y]), __uint_as_float(dv[x + y + 1])),
+                                         make_float2(-dl[y], -dl[y + 1]));
+            const float2 ds = __fmul2_rn(ps, in);
+            dsv[y] = ds.x;
+            dsv[y + 1] = ds.y;
+            pv[y] = ps.x * gp;                                      // g P, for dV
+            pv[y + 1] = ps.y * gp;
           }
           const __nv_bfloat162 a0 = __floats2bfloat162_rn(dsv[0], dsv[1]);
           const __nv_bfloat162 a1 = __floats2bfloat162_rn(dsv[2], dsv[3]);
