@@ -366,34 +366,27 @@ bwd_tc_kernel(const __grid_constant__ BwdTcParams p) {
       ok = __all_sync(0xffffffffu, ok);   // the tensor-memory accesses below are warp-collective
       if (C::kRowWgs == 1 && !ok) break;
       if (ok) tc_fence_after();
-      // visible columns of a row at slot rs: one interval [lo, hi], cut by the token order
+      // visible columns of this row: one interval [lo, lo + span], cut by the token order
       const int cb = cstart + j * KC;
-      auto interval = [&](int rs, int* lo_out, int* hi_out) {
-        int lo, hi;
-        if (p.one_sided) {
-          if (kKeys) { lo = rs - cb; hi = p.full_range ? p.n - 1 - cb : rs + (p.w - 1) - cb; }
-          else { lo = p.full_range ? -cb : rs - (p.w - 1) - cb; hi = rs - cb; }
-        } else if (p.full_range && !p.linear) { lo = -cb; hi = p.n - 1 - cb; }
-        else { lo = rs - p.h - cb; hi = rs + p.h - cb; }
-        if (p.linear || p.full_range || p.one_sided) {
-          lo = max(lo, -cb);
-          hi = min(hi, p.n - 1 - cb);
-        }
-        if (hi < lo) { lo = 1 << 30; hi = lo; }
-        *lo_out = lo;
-        *hi_out = hi;
-      };
+      const bool clamp = p.linear || p.full_range || p.one_sided;
       int lo, hi;
-      interval(rslot, &lo, &hi);
-      const uint32_t span = (uint32_t)(hi - lo);
+      if (p.one_sided) {
+        if (kKeys) { lo = rslot - cb; hi = p.full_range ? p.n - 1 - cb : rslot + (p.w - 1) - cb; }
+        else { lo = p.full_range ? -cb : rslot - (p.w - 1) - cb; hi = rslot - cb; }
+      } else if (p.full_range && !p.linear) { lo = -cb; hi = p.n - 1 - cb; }
+      else { lo = rslot - p.h - cb; hi = rslot + p.h - cb; }
       // Every row of the tile sees every column of this tile (up to the token order) when the
-      // last row's interval starts at or before column 0 and the first row's ends at or after
-      // the last column: then the per-element interval test is left out.
-      int lo_last, hi_last, lo_first, hi_first;
-      interval(r0 + kTile - 1, &lo_last, &hi_last);
-      interval(r0, &lo_first, &hi_first);
-      const bool interior = lo_last <= 0 && hi_first >= KC - 1 && hi_last >= KC - 1 &&
-                            lo_first <= 0 && r0 + kTile - 1 < p.n;
+      // last row's interval starts at or before column 0, the first row's ends at or after the
+      // last column and no clamp cuts in: then the per-element interval test is left out.
+      // (The interval moves with the row's slot, one column per row.)
+      const bool interior = !p.full_range && lo + (kTile - 1 - row) <= 0 && hi - row >= KC - 1 &&
+                            (!clamp || (cb >= 0 && cb + KC <= p.n)) && r0 + kTile - 1 < p.n;
+      if (clamp) {
+        lo = max(lo, -cb);
+        hi = min(hi, p.n - 1 - cb);
+      }
+      if (hi < lo) { lo = 1 << 30; hi = lo; }
+      const uint32_t span = (uint32_t)(hi - lo);
       const int32_t* coltok = reinterpret_cast<const int32_t*>(smem + C::kOffColTok) + s * kTile;
       const float* colvec = reinterpret_cast<const float*>(smem + C::kOffColVec) + s * 2 * kTile;
 #pragma unroll 1
