@@ -179,6 +179,9 @@ def main():
     ap.add_argument("--workload", default="C3")
     ap.add_argument("--n", type=int, default=0,
                     help="override the sequence length (profiling captures on a smaller case)")
+    ap.add_argument("--leg", default="step", choices=["step", "backward"],
+                    help="backward: time the gated backward of the workload instead of the step "
+                         "(a side measurement with its own JSON line; used for profiling)")
     ap.add_argument("--no-extras", action="store_true",
                     help="skip the side measurements (SWA, backward, e2e, CPU oracle)")
     args = ap.parse_args()
@@ -222,6 +225,10 @@ def main():
                                             sa.OP_GATED_FORWARD_SCRATCH),
                       dtype=torch.uint8, device="cuda")
     torch.cuda.synchronize()
+
+    if args.leg == "backward":
+        backward_leg(args, c, sa, torch, dev, perm, inv, ws, rank)
+        return
 
     layer = [0]
 
@@ -302,6 +309,33 @@ def main():
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def backward_leg(args, c, sa, torch, dev, perm, inv, ws, rank):
+    """Gated forward once (saving what the backward needs), then `steps` timed backward passes."""
+    q, k, v, lg = dev["q"], dev["k"], dev["v"], dev["gate_logits"]
+    dy = torch.randn(q.shape, generator=torch.Generator(device="cuda").manual_seed(c.seed + 77),
+                     device="cuda", dtype=torch.float32).to(q.dtype)
+    sa.sa_make_perm(c.seed, 0, c.B, c.n, perm=perm, inv=inv, ws=ws)
+    _, y_sa, y_swa, lse_sa, lse_swa = sa.sa_swa_gated_forward(q, k, v, perm, inv, lg, c.w, c.flags,
+                                                              save_for_bwd=True)
+    bws = torch.empty(sa.sa_workspace_bytes(sa.make_problem(q, k, c.w, c.flags), sa.OP_BACKWARD),
+                      dtype=torch.uint8, device="cuda")
+    out = {}
+
+    def bwd():
+        r = sa.sa_backward(q, k, v, perm, inv, lg, y_sa, y_swa, lse_sa, lse_swa, dy, c.w, c.flags,
+                           ws=bws, out=out)
+        out.update(zip(("dq", "dk", "dv", "dgate"), r))
+    ms = event_ms(bwd, args.steps, args.warmup, torch)
+    assert sa.sa_read_status() == 0
+    flops = 2 * 2.5 * 4.0 * c.B * c.Hq * c.n * c.w * c.d
+    if rank == 0:
+        print(json.dumps({"leg": "backward", "metric": "gated SA+SWA backward tokens/s",
+                          "value": c.B * c.n / (ms * 1e-3), "unit": "tokens/s", "ms_per_step": ms,
+                          "steps": args.steps, "warmup": args.warmup,
+                          "tflops_nominal": flops / (ms * 1e-3) / 1e12,
+                          "config": workload_config(c), "dtype": "bf16", "data": "synthetic"}))
 
 
 def extras(args, c, wl, sa, torch, dev, host, perm, inv, ws, y, pk):
