@@ -248,6 +248,37 @@ def forward_rows(swa, q, k, v, perm, inv, w, flags, rows, scale=0.0):
     return y, lse
 
 
+def backward_rows(q, k, v, perm, inv, gate_logits, dy, w, flags, q_rows, kv_rows, scale=0.0):
+    """Selected rows of the gradients of sum(dy*y) (same derivative as ``backward``).
+
+    q_rows: flat (b*Hq+hq)*n+i indices -> dq rows; kv_rows: flat (b*Hkv+hk)*n+j indices ->
+    dk and dv rows (summed over the group's query heads, the branches and every query that
+    sees the key).  gate_logits None => ungated SA only.  Returns (dq_rows, dk_rows, dv_rows)."""
+    q, qp = _f64(q)
+    k, kp = _f64(k)
+    v, vp = _f64(v)
+    dy, dyp = _f64(dy)
+    B, Hq, n, d = q.shape
+    Hkv = k.shape[1]
+    perm, pp = _i32(perm)
+    inv, ip = _i32(inv)
+    g, gp = (None, None) if gate_logits is None else _f64(gate_logits)
+    q_rows = np.ascontiguousarray(q_rows, dtype=np.int64)
+    kv_rows = np.ascontiguousarray(kv_rows, dtype=np.int64)
+    dq = np.empty((q_rows.size, d), np.float64)
+    dk = np.empty((kv_rows.size, d), np.float64)
+    dv = np.empty((kv_rows.size, d), np.float64)
+    _load().oracle_backward_rows(
+        ctypes.c_int32(B), ctypes.c_int32(Hq), ctypes.c_int32(Hkv), ctypes.c_int32(n),
+        ctypes.c_int32(d), ctypes.c_int32(w), ctypes.c_uint32(flags),
+        ctypes.c_double(_scale(d, scale)), qp, kp, vp, pp, ip, gp, dyp,
+        ctypes.c_int64(q_rows.size), q_rows.ctypes.data_as(ctypes.c_void_p),
+        dq.ctypes.data_as(ctypes.c_void_p),
+        ctypes.c_int64(kv_rows.size), kv_rows.ctypes.data_as(ctypes.c_void_p),
+        dk.ctypes.data_as(ctypes.c_void_p), dv.ctypes.data_as(ctypes.c_void_p))
+    return dq, dk, dv
+
+
 def gate_projection(y_sa, w_sa, y_swa=None, w_swa=None):
     """Projection gates of Eq. 5-6 (App. B, dual-path and single-path attention gate).
 

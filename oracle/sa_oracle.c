@@ -29,7 +29,10 @@
  * bijection/uniformity, closed-form mask counts, Prop. 1 by exhaustion, identity
  * permutation == independently written SWA, w >= n+1 == dense attention, Alg. 1
  * three-stage form, uniform-attention mean, w = 1 gives Y = V, finite differences
- * for every gradient, closed-form SWA reach.  No function here is unpinned.
+ * for every gradient, closed-form SWA reach; the selected-row variants
+ * (oracle_forward_rows, oracle_backward_rows) on every row index of small cases against
+ * the whole-tensor functions and against dense numpy attention.  No function here is
+ * unpinned.
  *
  * Layout: all tensors contiguous, q/y/dq [B,Hq,n,d], k/v/dk/dv [B,Hkv,n,d],
  * perm/inv [B,n], lse [B,Hq,n]; everything in ORIGINAL token order.
@@ -414,5 +417,104 @@ void oracle_forward_rows(int32_t swa, int32_t B, int32_t Hq, int32_t Hkv, int32_
       if (lse_rows) lse_rows[t] = l;
     }
     free(cand); free(s_buf);
+  }
+}
+
+/* Selected gradient rows only, for spot checks at sizes where oracle_backward would take
+ * days.  Same formulas as oracle_backward (textbook derivative of Eq. 1 / Eq. 5), written
+ * per requested row:
+ *   q_rows[t] = flat (b*Hq + hq)*n + i   ->  dq_rows[t][d]: sum over the branches x and the
+ *               keys j visible to query i of scale * dS_ij * K_j;
+ *   kv_rows[t] = flat (b*Hkv + hk)*n + j ->  dk_rows[t][d], dv_rows[t][d]: sum over the query
+ *               heads of the group, the branches and EVERY query token i that sees key j
+ *               (all n tokens are tested with the branch's predicate) of scale * dS_ij * Q_i
+ *               and P_ij * dY_x[i].
+ * Each query's softmax row is recomputed in full, as in oracle_backward.  gate_logits ==
+ * NULL: ungated SA only.                                                               */
+void oracle_backward_rows(int32_t B, int32_t Hq, int32_t Hkv, int32_t n, int32_t d, int32_t w,
+                          uint32_t flags, double scale, const double* q, const double* k,
+                          const double* v, const int32_t* perm, const int32_t* inv,
+                          const double* gate_logits, const double* dy,
+                          int64_t n_q_rows, const int64_t* q_rows, double* dq_rows,
+                          int64_t n_kv_rows, const int64_t* kv_rows, double* dk_rows,
+                          double* dv_rows) {
+  const int32_t G = Hq / Hkv;
+  const int32_t nbranch = gate_logits ? 2 : 1;
+  (void)B;
+#pragma omp parallel
+  {
+    int32_t* cand = (int32_t*)malloc(sizeof(int32_t) * (size_t)n);
+    double* p = (double*)malloc(sizeof(double) * (size_t)n);
+    double* yx = (double*)malloc(sizeof(double) * (size_t)d);
+    double* dyx = (double*)malloc(sizeof(double) * (size_t)d);
+#pragma omp for schedule(dynamic, 4)
+    for (int64_t t = 0; t < n_q_rows; ++t) {
+      const int64_t r = q_rows[t];
+      const int32_t i = (int32_t)(r % n);
+      const int32_t hq = (int32_t)((r / n) % Hq);
+      const int32_t b = (int32_t)(r / ((int64_t)n * Hq));
+      const int32_t hk = hq / G;
+      const int32_t* pb = perm ? perm + (size_t)b * n : NULL;
+      const int32_t* ib = inv ? inv + (size_t)b * n : NULL;
+      const double* kh = k + ((size_t)b * Hkv + hk) * n * d;
+      const double* vh = v + ((size_t)b * Hkv + hk) * n * d;
+      const double* qr = q + (size_t)r * d;
+      double* out = dq_rows + (size_t)t * d;
+      for (int32_t c = 0; c < d; ++c) out[c] = 0.0;
+      for (int32_t x = 0; x < nbranch; ++x) {
+        const double g = gate_logits ? sigmoid(gate_logits[x * Hq + hq]) : 1.0;
+        const int32_t nc = collect_visible(x == 1, 0, n, w, flags, pb, ib, i, cand);
+        attend_row(d, scale, qr, kh, vh, cand, nc, p, yx);
+        double D = 0.0;
+        for (int32_t c = 0; c < d; ++c) { dyx[c] = g * dy[(size_t)r * d + c]; D += dyx[c] * yx[c]; }
+        for (int32_t u = 0; u < nc; ++u) {
+          const int32_t j = cand[u];
+          double dp = 0.0;
+          for (int32_t c = 0; c < d; ++c) dp += dyx[c] * vh[(size_t)j * d + c];
+          const double ds = p[u] * (dp - D);
+          for (int32_t c = 0; c < d; ++c) out[c] += scale * ds * kh[(size_t)j * d + c];
+        }
+      }
+    }
+#pragma omp for schedule(dynamic, 1)
+    for (int64_t t = 0; t < n_kv_rows; ++t) {
+      const int64_t r = kv_rows[t];
+      const int32_t j = (int32_t)(r % n);
+      const int32_t hk = (int32_t)((r / n) % Hkv);
+      const int32_t b = (int32_t)(r / ((int64_t)n * Hkv));
+      const int32_t* pb = perm ? perm + (size_t)b * n : NULL;
+      const int32_t* ib = inv ? inv + (size_t)b * n : NULL;
+      const double* kh = k + ((size_t)b * Hkv + hk) * n * d;
+      const double* vh = v + ((size_t)b * Hkv + hk) * n * d;
+      double* odk = dk_rows + (size_t)t * d;
+      double* odv = dv_rows + (size_t)t * d;
+      for (int32_t c = 0; c < d; ++c) { odk[c] = 0.0; odv[c] = 0.0; }
+      for (int32_t hq = hk * G; hq < (hk + 1) * G; ++hq)
+        for (int32_t x = 0; x < nbranch; ++x) {
+          const double g = gate_logits ? sigmoid(gate_logits[x * Hq + hq]) : 1.0;
+          for (int32_t i = 0; i < n; ++i) {
+            if (!branch_visible(x == 1, n, w, flags, ib, i, j)) continue;
+            const size_t qi = ((size_t)b * Hq + hq) * n + i;
+            const double* qr = q + qi * d;
+            const int32_t nc = collect_visible(x == 1, 0, n, w, flags, pb, ib, i, cand);
+            attend_row(d, scale, qr, kh, vh, cand, nc, p, yx);
+            int32_t at = -1;
+            for (int32_t u = 0; u < nc; ++u) if (cand[u] == j) { at = u; break; }
+            if (at < 0) continue;   /* cannot happen: j passed the same predicate */
+            double D = 0.0, dp = 0.0;
+            for (int32_t c = 0; c < d; ++c) {
+              dyx[c] = g * dy[qi * d + c];
+              D += dyx[c] * yx[c];
+              dp += dyx[c] * vh[(size_t)j * d + c];
+            }
+            const double ds = p[at] * (dp - D);
+            for (int32_t c = 0; c < d; ++c) {
+              odv[c] += p[at] * dyx[c];
+              odk[c] += scale * ds * qr[c];
+            }
+          }
+        }
+    }
+    free(cand); free(p); free(yx); free(dyx);
   }
 }

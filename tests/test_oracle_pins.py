@@ -413,6 +413,114 @@ def test_backward_gqa_sums_group_and_equivariance():
     assert np.abs(dv3[:, :, inv[0]] - dv).max() < TOL
 
 
+# ------------------------------------------------------- selected-row variants
+
+ROW_CASES = [
+    # B, Hq, Hkv, n, d, w, flags
+    (2, 4, 2, 37, 8, 9, CAUSAL | SWA_ONE_SIDED),
+    (1, 6, 3, 50, 4, 16, 0),
+    (3, 2, 2, 24, 8, 64, CAUSAL),                 # window wider than the sequence
+    (2, 4, 1, 41, 4, 7, CAUSAL | LINEAR_WINDOW | SWA_ONE_SIDED),
+]
+
+
+def np_branch_mask(swa, inv, n, w, flags):
+    """Mask [query token, key token] of one branch, from the printed inequalities."""
+    if swa and flags & SWA_ONE_SIDED:
+        i = np.arange(n)
+        back = i[:, None] - i[None, :]
+        return (back >= 0) & (back <= w - 1)
+    slots = np.arange(n) if swa else inv
+    return np_mask_eq3(slots, n, w, bool(flags & CAUSAL), circular=not flags & LINEAR_WINDOW)
+
+
+@pytest.mark.parametrize("case", ROW_CASES)
+def test_forward_rows_equals_full_forward_on_every_row(case):
+    """Every flat row index, in shuffled order, against the whole-tensor functions (bitwise)
+    and against textbook dense attention written in numpy (independent of the oracle)."""
+    B, Hq, Hkv, n, d, w, flags = case
+    rng = np.random.default_rng(B * 100 + n)
+    q, k, v = qkv(rng, B, Hq, Hkv, n, d)
+    perm, inv = rand_perm(rng, B, n)
+    rows = rng.permutation(B * Hq * n).astype(np.int64)
+    G = Hq // Hkv
+    scale = 1.0 / math.sqrt(d)
+    for swa in (0, 1):
+        full_y, full_lse = (oracle.swa_forward(q, k, v, w, flags) if swa
+                            else oracle.sa_forward(q, k, v, perm, inv, w, flags))
+        y, lse = oracle.forward_rows(swa, q, k, v, perm, inv, w, flags, rows)
+        assert np.array_equal(y, full_y.reshape(-1, d)[rows])
+        assert np.array_equal(lse, full_lse.reshape(-1)[rows])
+        # the row decoding r -> (b, hq, i) and hq -> hk, against numpy dense attention
+        for t in rng.choice(rows.size, size=25, replace=False):
+            r = int(rows[t])
+            i, hq, b = r % n, (r // n) % Hq, r // (n * Hq)
+            mask = np_branch_mask(swa, inv[b], n, w, flags)
+            ry, rl = np_dense_attention(q[b, hq], k[b, hq // G], v[b, hq // G], mask, scale)
+            assert np.abs(y[t] - ry[i]).max() < TOL and abs(lse[t] - rl[i]) < TOL
+    # duplicates and an empty request
+    y, lse = oracle.forward_rows(0, q, k, v, perm, inv, w, flags, [5, 5, 0])
+    assert np.array_equal(y[0], y[1]) and y.shape == (3, d)
+    y, lse = oracle.forward_rows(0, q, k, v, perm, inv, w, flags, [])
+    assert y.shape == (0, d) and lse.shape == (0,)
+
+
+def np_dense_backward(q, k, v, inv, lg, dy, w, flags):
+    """Textbook gradients of sum(dy*y) with dense n x n matrices, numpy only.
+    P = softmax(mask(S)), dV = P^T dY, dS = P o (dY V^T - rowsum(dY o Y)), dQ = scale dS K,
+    dK = scale dS^T Q; both branches through Eq. 5 when lg is given."""
+    B, Hq, n, d = q.shape
+    Hkv = k.shape[1]
+    G = Hq // Hkv
+    scale = 1.0 / math.sqrt(d)
+    dq, dk, dv = np.zeros_like(q), np.zeros_like(k), np.zeros_like(v)
+    for b in range(B):
+        for hq in range(Hq):
+            hk = hq // G
+            for x in range(2 if lg is not None else 1):
+                g = 1.0 if lg is None else 1.0 / (1.0 + math.exp(-lg[x, hq]))
+                mask = np_branch_mask(x, inv[b], n, w, flags)
+                s = np.where(mask, (q[b, hq] @ k[b, hk].T) * scale, -np.inf)
+                p = np.exp(s - s.max(axis=1, keepdims=True))
+                p /= p.sum(axis=1, keepdims=True)
+                dyx = g * dy[b, hq]
+                yx = p @ v[b, hk]
+                ds = p * (dyx @ v[b, hk].T - (dyx * yx).sum(axis=1, keepdims=True))
+                dv[b, hk] += p.T @ dyx
+                dq[b, hq] += scale * ds @ k[b, hk]
+                dk[b, hk] += scale * ds.T @ q[b, hq]
+    return dq, dk, dv
+
+
+@pytest.mark.parametrize("gated", [False, True])
+@pytest.mark.parametrize("case", ROW_CASES)
+def test_backward_rows_equals_full_backward_on_every_row(case, gated):
+    B, Hq, Hkv, n, d, w, flags = case
+    rng = np.random.default_rng(B * 100 + n + gated)
+    q, k, v = qkv(rng, B, Hq, Hkv, n, d)
+    dy = rng.standard_normal(q.shape)
+    perm, inv = rand_perm(rng, B, n)
+    lg = rng.standard_normal((2, Hq)) if gated else None
+    dq, dk, dv, _ = oracle.backward(q, k, v, perm, inv, lg, dy, w, flags)
+    # the whole-tensor backward itself against dense numpy matrices (not the oracle)
+    ndq, ndk, ndv = np_dense_backward(q, k, v, inv, lg, dy, w, flags)
+    for a, b_ in ((dq, ndq), (dk, ndk), (dv, ndv)):
+        assert np.abs(a - b_).max() < 1e-11 * max(1.0, np.abs(b_).max())
+    q_rows = rng.permutation(B * Hq * n).astype(np.int64)
+    kv_rows = rng.permutation(B * Hkv * n).astype(np.int64)
+    rdq, rdk, rdv = oracle.backward_rows(q, k, v, perm, inv, lg, dy, w, flags, q_rows, kv_rows)
+    for got, want in ((rdq, ndq.reshape(-1, d)[q_rows]), (rdk, ndk.reshape(-1, d)[kv_rows]),
+                      (rdv, ndv.reshape(-1, d)[kv_rows])):
+        assert np.abs(got - want).max() < 1e-11 * max(1.0, np.abs(want).max())
+    for got, want in ((rdq, dq.reshape(-1, d)[q_rows]), (rdk, dk.reshape(-1, d)[kv_rows]),
+                      (rdv, dv.reshape(-1, d)[kv_rows])):
+        assert np.abs(got - want).max() < 1e-12 * max(1.0, np.abs(want).max())
+    # one list may be empty
+    a, b_, c = oracle.backward_rows(q, k, v, perm, inv, lg, dy, w, flags, [3], [])
+    assert a.shape == (1, d) and b_.shape == (0, d) and c.shape == (0, d)
+    assert np.array_equal(a[0], rdq[list(q_rows).index(3)])
+
+
 # ------------------------------------------------------------------- coverage
 
 def test_swa_reach_closed_form():
