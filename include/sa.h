@@ -31,7 +31,9 @@
  *     workspace) return a code before anything is launched.  Errors only the device can
  *     see (SA_VALIDATE_PERM found a non-bijection, a bounded wait ran out) are recorded
  *     in a device status word that sa_read_status returns; the kernel then returns
- *     normally and its outputs are unspecified.  Nothing traps.
+ *     normally and its outputs are unspecified.  Nothing traps.  The word is sticky: once
+ *     it holds SA_ERR_TIMEOUT, later tensor-core launches return at once without writing
+ *     their outputs until sa_read_status has been called (which clears it).
  */
 #ifndef SA_B200_SA_H_
 #define SA_B200_SA_H_
@@ -234,6 +236,35 @@ void sa_set_profile_events(void* start, void* stop);
 /* Number of kernel launches this process has enqueued through the library so far
  * (all entry points together); used by the benchmark's launch count. */
 uint64_t sa_launch_count(void);
+
+/* Test hooks.  The library reads no environment variable; these process-wide switches exist
+ * so that tests can run every kernel variant on one input.  The paper has no counterpart.
+ *   SA_DEBUG_SCORE_BLOCK      0 = choose by w (default), 64 or 128 = force that score-block
+ *                             width in the tensor-core forward and the matching backward shape
+ *   SA_DEBUG_SWA_TILE_LOADS   1 = one-sided SWA branch loads whole tiles by TMA when the layout
+ *                             allows (default), 0 = always gather rows
+ *   SA_DEBUG_TENSOR_CORES     1 = tensor-core kernels where they apply (default), 0 = the
+ *                             general CUDA-core kernels everywhere
+ *   SA_DEBUG_GATE_WIDE_TILES  1 = 128 x 256 tiles for large gate projections (default), 0 = the
+ *                             fused 128 x 128 kernel
+ * Returns SA_ERR_INVALID_ARG for an unknown key or value.  Takes effect for later calls. */
+typedef enum {
+  SA_DEBUG_SCORE_BLOCK = 0,
+  SA_DEBUG_SWA_TILE_LOADS = 1,
+  SA_DEBUG_TENSOR_CORES = 2,
+  SA_DEBUG_GATE_WIDE_TILES = 3,
+  SA_DEBUG_KEYS = 4
+} sa_debug_key;
+sa_status sa_debug_set(int key, int value);
+
+/* Test hook for the failure path of the kernels' bounded waits.  Launches one small CTA on
+ * `stream` that waits, with the same wait routine the attention kernels use, on a barrier that
+ * nothing ever completes, for at most limit_cycles SM clock cycles (1 .. 2^31; a million is
+ * about half a millisecond).  The wait gives up, records SA_ERR_TIMEOUT in the device status
+ * word and the kernel returns normally: nothing traps, faults or spins without a bound.
+ * While the status word holds SA_ERR_TIMEOUT every tensor-core kernel of the library returns
+ * at once without writing its outputs; sa_read_status returns the code and clears it. */
+sa_status sa_debug_wait_timeout(int64_t limit_cycles, sa_stream_t stream);
 
 #ifdef __cplusplus
 }

@@ -29,8 +29,9 @@ EXPORTS = [
     "sa_swa_forward", "sa_swa_gated_forward", "sa_backward", "sa_coverage", "sa_read_status",
     "sa_status_string", "sa_launch_count", "sa_set_profile_events", "sa_make_perm_static",
     "sa_gate_projection_forward", "sa_gate_projection_backward",
-    "sa_gate_projection_backward_ws_bytes",
+    "sa_gate_projection_backward_ws_bytes", "sa_debug_set", "sa_debug_wait_timeout",
 ]
+DEBUG_SCORE_BLOCK, DEBUG_SWA_TILE_LOADS, DEBUG_TENSOR_CORES, DEBUG_GATE_WIDE_TILES = range(4)
 
 
 class SaProblem(ctypes.Structure):
@@ -63,9 +64,10 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
             try:
                 _build.build_library()
             except Exception as e:  # no nvcc, compile error
-                if not os.path.exists(path):
-                    raise RuntimeError("CUDA library %s is missing and could not be built: %s"
-                                       % (path, e)) from e
+                # never run a library older than its sources: that would test stale kernels
+                what = "is older than its sources" if os.path.exists(path) else "is missing"
+                raise RuntimeError("CUDA library %s %s and could not be built: %s"
+                                   % (path, what, e)) from e
     lib = ctypes.CDLL(path)
     vp, i32, u32, u64, sz = (ctypes.c_void_p, ctypes.c_int32, ctypes.c_uint32, ctypes.c_uint64,
                              ctypes.c_size_t)
@@ -101,6 +103,10 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.sa_set_profile_events.restype = None
     lib.sa_launch_count.argtypes = []
     lib.sa_launch_count.restype = u64
+    lib.sa_debug_set.argtypes = [ctypes.c_int, ctypes.c_int]
+    lib.sa_debug_set.restype = ctypes.c_int
+    lib.sa_debug_wait_timeout.argtypes = [i64, vp]
+    lib.sa_debug_wait_timeout.restype = ctypes.c_int
     if path == _build.LIB:
         _lib = lib
     return lib
@@ -126,6 +132,17 @@ def set_profile_events(start: Optional[torch.cuda.Event], stop: Optional[torch.c
     if not stop.cuda_event:
         stop.record()
     lib.sa_set_profile_events(ctypes.c_void_p(start.cuda_event), ctypes.c_void_p(stop.cuda_event))
+
+
+def debug_set(key: int, value: int):
+    """Test hook: selects a kernel variant for later calls (see sa_debug_set in sa.h)."""
+    _check(load_library().sa_debug_set(int(key), int(value)), "sa_debug_set")
+
+
+def debug_wait_timeout(limit_cycles: int):
+    """Test hook: one small kernel whose bounded wait runs out after limit_cycles."""
+    _check(load_library().sa_debug_wait_timeout(int(limit_cycles), _stream()),
+           "sa_debug_wait_timeout")
 
 
 def _ptr(t: Optional[torch.Tensor]):

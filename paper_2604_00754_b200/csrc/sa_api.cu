@@ -14,16 +14,23 @@ static cudaEvent_t g_prof_start = nullptr, g_prof_stop = nullptr;
 
 void bump_launches(uint64_t k) { g_launches.fetch_add(k, std::memory_order_relaxed); }
 
+// Test hooks: score block auto, SWA tile loads on, tensor cores on, wide gate tiles on.
+static std::atomic<int> g_debug[SA_DEBUG_KEYS] = {{0}, {1}, {1}, {1}};
+
+int debug_option(int key) {
+  return key >= 0 && key < SA_DEBUG_KEYS ? g_debug[key].load(std::memory_order_relaxed) : 0;
+}
+
 int* status_ptr() {
-  static int* ptrs[64] = {nullptr};
+  static std::atomic<int*> ptrs[64];
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-  if (!ptrs[dev]) {
-    int* p = nullptr;
+  int* p = ptrs[dev].load(std::memory_order_acquire);
+  if (!p) {
     if (cudaGetSymbolAddress((void**)&p, g_status_word) != cudaSuccess) return nullptr;
-    ptrs[dev] = p;
+    ptrs[dev].store(p, std::memory_order_release);
   }
-  return ptrs[dev];
+  return p;
 }
 
 namespace {
@@ -305,5 +312,14 @@ void sa_set_profile_events(void* start, void* stop) {
 }
 
 uint64_t sa_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+sa_status sa_debug_set(int key, int value) {
+  if (key < 0 || key >= SA_DEBUG_KEYS) return SA_ERR_INVALID_ARG;
+  if (key == SA_DEBUG_SCORE_BLOCK ? (value != 0 && value != 64 && value != 128)
+                                  : (value != 0 && value != 1))
+    return SA_ERR_INVALID_ARG;
+  g_debug[key].store(value, std::memory_order_relaxed);
+  return SA_OK;
+}
 
 }  // extern "C"

@@ -120,8 +120,9 @@ bwd_tc_kernel(const __grid_constant__ BwdTcParams p) {
   constexpr bool kKeys = MODE == 1;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-  if (p.abort_flag && *p.abort_flag) return;  // an earlier check rejected perm/inv (uniform)
-  if (*(volatile int*)p.status == SA_ERR_TIMEOUT) return;
+  if (cta_should_skip(reinterpret_cast<volatile int*>(smem + C::kOffMisc + 8), p.status,
+                      p.abort_flag))
+    return;
   const uint32_t sbase = smem_u32(smem);
   if (sbase & 1023u) {
     if (threadIdx.x == 0) atomicCAS(p.status, SA_OK, SA_ERR_CUDA);
@@ -534,25 +535,14 @@ cudaError_t launch_branch(const BwdTcParams& p, cudaStream_t st) {
 // Kernel shape: 0 = 64-wide column tiles, one score buffer (narrow windows: least band-edge
 // waste, two CTAs per SM at d = 64); 1 = 64-wide tiles, two score buffers and two row
 // warpgroups (products of the next tile overlap the row work of this one); 2 = 128-wide
-// tiles, one buffer.  SA_KEY_BLOCK=64|128 forces shape 0 or 2 so tests can run every shape.
+// tiles, one buffer.  sa_debug_set(SA_DEBUG_SCORE_BLOCK, 64 | 128) forces shape 0 or 2.
 int bwd_shape(int w) {
-  static int forced = -1;
-  if (forced < 0) {
-    const char* e = getenv("SA_KEY_BLOCK");
-    forced = !e ? 0 : (e[0] == '6' ? 64 : 128);
-  }
+  const int forced = debug_option(SA_DEBUG_SCORE_BLOCK);
   if (forced) return forced == 64 ? 0 : 2;
   return w <= 128 ? 0 : 1;
 }
 
-bool bwd_tc_disabled() {
-  static int v = -1;
-  if (v < 0) {
-    const char* e = getenv("SA_DISABLE_TC");
-    v = (e && e[0] == '1') ? 1 : 0;
-  }
-  return v == 1;
-}
+bool bwd_tc_disabled() { return debug_option(SA_DEBUG_TENSOR_CORES) == 0; }
 
 }  // namespace
 

@@ -109,6 +109,8 @@ __device__ __forceinline__ float warp_sum(float v) {
 // null if the runtime call that resolves it failed.
 int* status_ptr();
 void bump_launches(uint64_t k = 1);
+// Current value of a test hook (sa_debug_key); see sa_debug_set.
+int debug_option(int key);
 
 struct FwdArgs {
   const void *q, *k, *v;

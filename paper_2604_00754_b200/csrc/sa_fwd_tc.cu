@@ -52,10 +52,8 @@ struct TcParams {
   const int* abort_flag;
   int B, Hq, Hkv, G, n, w, h;
   int causal, linear, one_sided, swa, full_range;
-  // One-sided SWA branch on tensors that are plain 2-D matrices of rows: whole tiles come
-  // by TMA (row of (b, h, token) = b * rb + h * rh + token, first column h * ch)
+  // One-sided SWA branch: whole tiles come by TMA through rank-4 maps (d, token, head, batch)
   int use_tma;
-  int64_t q_rb, q_rh, q_ch, k_rb, k_rh, k_ch;
   int pair_heads;             // 1: tiles = two heads, same slots; 0: two slot tiles, one head
   int n_tiles;                // slot tiles of 128
   int items_per_kv;           // work items per (b, hk)
@@ -204,10 +202,9 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
   constexpr int kShift = KB == 64 ? 6 : 7;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-  if (p.abort_flag && *p.abort_flag) return;  // an earlier check rejected perm/inv (uniform)
-  // Once any CTA has recorded a timeout the rest of the grid leaves at once instead of
-  // each waiting out its own limit.
-  if (*(volatile int*)p.status == SA_ERR_TIMEOUT) return;
+  if (cta_should_skip(reinterpret_cast<volatile int*>(smem + C::kOffMisc + 8), p.status,
+                      p.abort_flag))
+    return;
   const uint32_t sbase = smem_u32(smem);
   if (sbase & 1023u) {                        // the swizzled tiles need 1024-byte alignment
     if (threadIdx.x == 0) atomicCAS(p.status, SA_OK, SA_ERR_CUDA);
@@ -246,26 +243,26 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
   asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
   if (warp >= 1 && TMA) {
     // ------------------------------------------- tile loads by TMA (one thread of warp 1)
-    // Rows are consecutive tokens here, so a tile is D / 64 boxes of 128 rows x 64 columns
+    // Rows are consecutive tokens here, so a tile is D / 64 boxes of 128 tokens x 64 columns
     // that the TMA unit lays out in the same swizzled form the gather produces; no producer
-    // instructions compete with the softmax warps.  Rows past the sequence read the next
-    // rows of the matrix (or zeros past its end); the window mask never lets them count and
-    // their outputs are not stored.  The key-token lists are not written: the one-sided
-    // rule tests slots only.
+    // instructions compete with the softmax warps.  The token index is a dimension of the
+    // map, so rows past the sequence are filled with zeros (never with whatever follows in
+    // memory, which could be NaN and would poison P V through 0 * NaN); the window mask
+    // does not let them count and their outputs are not stored.  The key-token lists are
+    // not written: the one-sided rule tests slots only.
     if (threadIdx.x == 32) {
       uint32_t use = 0, gt = 0, it = 0, q_armed = 0xffffffffu;
       bool live = true;
-      auto load_tile = [&](const CUtensorMap* tm, uint32_t dst, int col, int64_t row, uint32_t mb) {
+      auto load_tile = [&](const CUtensorMap* tm, uint32_t dst, int tok, int head, int b,
+                           uint32_t mb) {
 #pragma unroll
         for (int c = 0; c < D / 64; ++c)
-          tma_load_2d(dst + c * C::kChunkBytes, tm, col + 64 * c, (int)row, mb);
+          tma_load_4d(dst + c * C::kChunkBytes, tm, 64 * c, tok, head, b, mb);
       };
       for (int w_item = blockIdx.x; w_item < p.total_items && live; w_item += gridDim.x, ++it) {
         const int item = w_item % p.items_per_kv, bh = w_item / p.items_per_kv;
         const int hk = bh % p.Hkv, b = bh / p.Hkv;
         const Geo g = make_geo(p, item, hk);
-        const int64_t krow = b * p.k_rb + hk * p.k_rh + g.kstart;
-        const int kcol = (int)(hk * p.k_ch);
         for (int j = 0; j < g.T; ++j, ++gt) {
           if (use >= (uint32_t)C::kSlots)
             live = mbar_wait(bar(C::kBarSlotEmpty + use % C::kSlots), (use / C::kSlots - 1) & 1u,
@@ -274,8 +271,8 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
           mbar_arrive(bar(C::kBarTokFull + gt % C::kTok));
           uint32_t mb = bar(C::kBarSlotFull + use % C::kSlots);
           mbar_expect_tx(mb, C::kTileBytes);
-          load_tile(&tm_k, sbase + C::kOffRing + (use % C::kSlots) * C::kTileBytes, kcol,
-                    krow + j * kTile, mb);
+          load_tile(&tm_k, sbase + C::kOffRing + (use % C::kSlots) * C::kTileBytes,
+                    g.kstart + j * kTile, hk, b, mb);
           ++use;
           if (j == 0) {
             if (it) live = mbar_wait(bar(C::kBarQEmpty), (it - 1) & 1u, gave_up, p.status);
@@ -284,8 +281,8 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
             q_armed = it;
 #pragma unroll
             for (int t = 0; t < 2; ++t)
-              load_tile(&tm_q, sbase + C::kOffQ + t * C::kTileBytes, (int)(g.hq[t] * p.q_ch),
-                        b * p.q_rb + g.hq[t] * p.q_rh + g.q0[t], bar(C::kBarQFull));
+              load_tile(&tm_q, sbase + C::kOffQ + t * C::kTileBytes, g.q0[t], g.hq[t], b,
+                        bar(C::kBarQFull));
           }
           if (use >= (uint32_t)C::kSlots)
             live = mbar_wait(bar(C::kBarSlotEmpty + use % C::kSlots), (use / C::kSlots - 1) & 1u,
@@ -293,8 +290,8 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
           if (!live) break;
           mb = bar(C::kBarSlotFull + use % C::kSlots);
           mbar_expect_tx(mb, C::kTileBytes);
-          load_tile(&tm_v, sbase + C::kOffRing + (use % C::kSlots) * C::kTileBytes, kcol,
-                    krow + j * kTile, mb);
+          load_tile(&tm_v, sbase + C::kOffRing + (use % C::kSlots) * C::kTileBytes,
+                    g.kstart + j * kTile, hk, b, mb);
           ++use;
         }
       }
@@ -817,56 +814,17 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
 
 // Score-block width.  Narrow windows skip more with 64-key blocks; from w = 256 on the
 // 128-key block wins (half as many products, commits and softmax rounds per key).  The
-// environment variable SA_KEY_BLOCK=64|128 overrides the choice so tests can run both.
+// test hook sa_debug_set(SA_DEBUG_SCORE_BLOCK, 64 | 128) overrides the choice.
 bool key_block_128(int w) {
-  static int forced = -1;
-  if (forced < 0) {
-    const char* e = getenv("SA_KEY_BLOCK");
-    forced = !e ? 0 : (e[0] == '6' ? 64 : 128);
-  }
+  const int forced = debug_option(SA_DEBUG_SCORE_BLOCK);
   return forced ? forced == 128 : w > 128;
 }
 
-// SA_SWA_TMA=0 keeps the cp.async gather for the one-sided SWA branch too (tests run both).
-bool swa_tma_disabled() {
-  static int v = -1;
-  if (v < 0) {
-    const char* e = getenv("SA_SWA_TMA");
-    v = (e && e[0] == '0') ? 1 : 0;
-  }
-  return v == 1;
-}
+// sa_debug_set(SA_DEBUG_SWA_TILE_LOADS, 0) keeps the cp.async gather for the one-sided SWA
+// branch too.
+bool swa_tma_disabled() { return debug_option(SA_DEBUG_SWA_TILE_LOADS) == 0; }
 
-// Row (b, h, token) of a tensor with element strides s[0..2] as row b * rb + h * rh + token
-// and first column h * ch of one 2-D matrix with pitch s[2]; false when the layout is not of
-// that kind.  Also gives the matrix extent.
-bool row_view(const int64_t s[3], int B, int H, int n, int d, int64_t* rb, int64_t* rh,
-              int64_t* ch, int64_t* rows, int64_t* cols) {
-  const int64_t ts = s[2];
-  if (ts < d || s[0] % ts != 0) return false;
-  *rb = s[0] / ts;
-  if (s[1] % ts == 0) {
-    *rh = s[1] / ts;
-    *ch = 0;
-    *cols = d;
-  } else {
-    if (s[1] * (H - 1) + d > ts) return false;
-    *rh = 0;
-    *ch = s[1];
-    *cols = s[1] * (H - 1) + d;
-  }
-  *rows = (B - 1) * *rb + (H - 1) * *rh + n;
-  return *rows < (1ll << 31) - 4 * kTile;
-}
-
-bool tc_disabled() {
-  static int v = -1;
-  if (v < 0) {
-    const char* e = getenv("SA_DISABLE_TC");
-    v = (e && e[0] == '1') ? 1 : 0;
-  }
-  return v == 1;
-}
+bool tc_disabled() { return debug_option(SA_DEBUG_TENSOR_CORES) == 0; }
 
 }  // namespace
 
@@ -908,16 +866,14 @@ cudaError_t launch_fwd_tc(const FwdArgs& a, cudaStream_t st) {
   }
   const unsigned grid = (unsigned)min(p.total_items, sm_count[dev]);
   const bool wide = key_block_128(a.w);
-  // whole-tile TMA loads for the one-sided SWA branch when q and k/v are plain row matrices
+  // whole-tile TMA loads for the one-sided SWA branch (any strides the maps can express;
+  // otherwise the gather serves this branch too)
   CUtensorMap tm_q{}, tm_k{}, tm_v{};
   if (a.swa && mg.one_sided && !swa_tma_disabled()) {
-    int64_t qrows, qcols, krows, kcols;
-    if (row_view(a.qs, a.B, a.Hq, a.n, a.d, &p.q_rb, &p.q_rh, &p.q_ch, &qrows, &qcols) &&
-        row_view(a.ks, a.B, a.Hkv, a.n, a.d, &p.k_rb, &p.k_rh, &p.k_ch, &krows, &kcols) &&
-        aligned16(a.q) && aligned16(a.k) && aligned16(a.v) &&
-        make_map(&tm_q, a.q, qrows, qcols, a.qs[2], kTile) &&
-        make_map(&tm_k, a.k, krows, kcols, a.ks[2], kTile) &&
-        make_map(&tm_v, a.v, krows, kcols, a.ks[2], kTile))
+    if (aligned16(a.q) && aligned16(a.k) && aligned16(a.v) &&
+        make_map_bhnd(&tm_q, a.q, a.B, a.Hq, a.n, a.d, a.qs) &&
+        make_map_bhnd(&tm_k, a.k, a.B, a.Hkv, a.n, a.d, a.ks) &&
+        make_map_bhnd(&tm_v, a.v, a.B, a.Hkv, a.n, a.d, a.ks))
       p.use_tma = 1;
   }
   auto go = [&](auto kernel, int smem) {

@@ -74,7 +74,8 @@ gate_bwd_kernel(const __grid_constant__ BwdGateParams p, const __grid_constant__
   constexpr int kBlock = 2048 / TN;       // column tiles per block of the tile order
   extern __shared__ __align__(1024) uint8_t smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (*(volatile int*)p.status == SA_ERR_TIMEOUT) return;
+  if (cta_should_skip(reinterpret_cast<volatile int*>(smem + kOffMisc + 8), p.status, nullptr))
+    return;
   const uint32_t sbase = smem_u32(smem);
   if (sbase & 1023u) {
     if (threadIdx.x == 0) atomicCAS(p.status, SA_OK, SA_ERR_CUDA);
@@ -418,11 +419,7 @@ extern "C" sa_status sa_gate_projection_backward(
   if (ws_bytes < sa_gate_projection_backward_ws_bytes(rows, dm)) return SA_ERR_WORKSPACE;
   if (rows * (int64_t)dm > (1ll << 40)) return SA_ERR_UNSUPPORTED;
   cudaStream_t st = (cudaStream_t)stream;
-  static int tc_off = -1;
-  if (tc_off < 0) {
-    const char* e = getenv("SA_DISABLE_TC");
-    tc_off = (e && e[0] == '1') ? 1 : 0;
-  }
+  const bool tc_off = debug_option(SA_DEBUG_TENSOR_CORES) == 0;
   bool tc = !tc_off && dtype == SA_BF16 && dm % 64 == 0 && ld_y % 8 == 0 && ld_dout % 8 == 0 &&
             ld_dy % 8 == 0 && rows < (1ll << 31) - 256 && aligned16(ws) && aligned16(dout);
   const void* ptrs[] = {y_sa, w_sa, dy_sa, dw_sa, y_swa, w_swa, dy_swa, dw_swa};

@@ -58,7 +58,8 @@ gate_tc_kernel(const __grid_constant__ GateParams p, const __grid_constant__ CUt
                const __grid_constant__ CUtensorMap tm_wswa) {
   extern __shared__ __align__(1024) uint8_t smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (*(volatile int*)p.status == SA_ERR_TIMEOUT) return;
+  if (cta_should_skip(reinterpret_cast<volatile int*>(smem + kOffMisc + 8), p.status, nullptr))
+    return;
   const uint32_t sbase = smem_u32(smem);
   if (sbase & 1023u) {                        // the swizzled tiles need 1024-byte alignment
     if (threadIdx.x == 0) atomicCAS(p.status, SA_OK, SA_ERR_CUDA);
@@ -277,23 +278,16 @@ extern "C" sa_status sa_gate_projection_forward(int64_t rows, int32_t dm, int32_
   if (dtype != SA_F32 && dtype != SA_BF16) return SA_ERR_INVALID_ARG;
   if (rows * (int64_t)dm > (1ll << 40)) return SA_ERR_UNSUPPORTED;
   cudaStream_t st = (cudaStream_t)stream;
-  static int tc_off = -1;
-  if (tc_off < 0) {
-    const char* e = getenv("SA_DISABLE_TC");
-    tc_off = (e && e[0] == '1') ? 1 : 0;
-  }
+  const bool tc_off = debug_option(SA_DEBUG_TENSOR_CORES) == 0;
   const bool tc = !tc_off && dtype == SA_BF16 && dm % 64 == 0 && ld_y % 8 == 0 && ld_out % 8 == 0 &&
                   aligned16(y_sa) && aligned16(w_sa) && aligned16(out) &&
                   (!y_swa || (aligned16(y_swa) && aligned16(w_swa))) &&
                   rows < (1ll << 31) - 128;
   // Large products run one 128 x 256-tile launch per path (a quarter fewer operand bytes per
   // flop; the second path adds to the rounded result of the first); the fused dual-accumulator
-  // kernel below serves the rest, and everything with SA_GATE_WIDE=0 (tests run both).
-  static int wide_on = -1;
-  if (wide_on < 0) {
-    const char* e = getenv("SA_GATE_WIDE");
-    wide_on = (e && e[0] == '0') ? 0 : 1;
-  }
+  // kernel below serves the rest, and everything after
+  // sa_debug_set(SA_DEBUG_GATE_WIDE_TILES, 0).
+  const bool wide_on = debug_option(SA_DEBUG_GATE_WIDE_TILES) != 0;
   if (tc && wide_on) {
     int dev = 0, sms = 0;
     int* status = status_ptr();

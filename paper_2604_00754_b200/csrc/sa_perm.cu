@@ -1,6 +1,8 @@
 // Permutation generation (Alg. 1 line 1): Philox4x32-10 sort keys, a segmented sort by
 // (key, token) with one segment per sequence -- one radix pass on the leading key bits,
 // then ranking inside each bucket -- and the inverse written with the permutation.
+#include <atomic>
+
 #include "sa_common.cuh"
 
 namespace sa {
@@ -147,15 +149,15 @@ static __device__ __align__(256) unsigned char g_static_scratch[SA_STATIC_SCRATC
 
 // Device address of g_static_scratch on the current device, resolved once per device.
 unsigned char* static_scratch_ptr() {
-  static unsigned char* ptrs[64] = {nullptr};
+  static std::atomic<unsigned char*> ptrs[64];
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-  if (!ptrs[dev]) {
-    unsigned char* q = nullptr;
+  unsigned char* q = ptrs[dev].load(std::memory_order_acquire);
+  if (!q) {
     if (cudaGetSymbolAddress((void**)&q, g_static_scratch) != cudaSuccess) return nullptr;
-    ptrs[dev] = q;
+    ptrs[dev].store(q, std::memory_order_release);
   }
-  return ptrs[dev];
+  return q;
 }
 
 }  // namespace

@@ -46,18 +46,32 @@ __device__ __forceinline__ bool mbar_try_parked(uint32_t bar, uint32_t parity, u
   return ok != 0;
 }
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* gave_up,
-                                          int* status) {
+                                          int* status, long long limit = kWaitCycles) {
   if (mbar_try(bar, parity)) return true;
   const long long t0 = clock64();
   while (true) {
     if (mbar_try_parked(bar, parity, 2000u)) return true;
     if (*gave_up) return false;
-    if (clock64() - t0 > kWaitCycles) {
+    if (clock64() - t0 > limit) {
       *gave_up = 1;
       atomicCAS(status, SA_OK, SA_ERR_TIMEOUT);
       return false;
     }
   }
+}
+
+// Should this CTA leave before doing anything?  Yes when an earlier check rejected perm/inv
+// (abort_flag) or some CTA has already recorded a timeout: the rest of the grid then leaves at
+// once instead of each waiting out its own limit.  Thread 0 reads the words once and the CTA
+// agrees through `slot` (an int in shared memory), so the answer is the same for every thread
+// even if another kernel writes the status word at that moment.  Contains a __syncthreads.
+__device__ __forceinline__ bool cta_should_skip(volatile int* slot, const int* status,
+                                                const int* abort_flag) {
+  if (threadIdx.x == 0)
+    *slot = (abort_flag && *(volatile const int*)abort_flag) ||
+            *(volatile const int*)status == SA_ERR_TIMEOUT;
+  __syncthreads();
+  return *slot != 0;
 }
 
 // Orders shared-memory writes made through the generic proxy (cp.async) that this thread

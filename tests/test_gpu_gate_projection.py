@@ -53,16 +53,38 @@ def test_plain_path_odd_sizes(dtype, tol):
     _check(out, ya, wa, yb, wb, dm, tol)
 
 
-def test_model_width_sampled_rows():
+def _model_width_rows(rows, rng):
+    """>= 512 random rows plus every row of the first and of the last 128-row tile."""
+    idx = np.unique(np.concatenate([rng.choice(rows, size=512, replace=False),
+                                    np.arange(0, 128), np.arange(rows - 128, rows)]))
+    return torch.from_numpy(idx)
+
+
+@pytest.mark.parametrize("wide", [True, False])
+@pytest.mark.parametrize("dual", [True, False])
+def test_model_width_sampled_rows(wide, dual):
     """Qwen3-8B width (Hq*d = 4096) on the attention output layout [B,n,Hq,d] viewed as
-    [B*n, Hq*d]; sampled rows against the oracle."""
+    [B*n, Hq*d].  wide: the 128 x 256-tile kernel the library picks at this size (dual path:
+    second launch accumulates into the rounded result of the first); not wide: the fused
+    128 x 128 kernel forced at the same size through the test hook."""
     from paper_2604_00754_b200 import binding as sa
     rows, dm = 4096, 4096
     ya, yb, wa, wb = _draw(rows, dm, 9, torch.bfloat16)
-    out = sa.sa_gate_projection_forward(ya.cuda(), wa.cuda(), yb.cuda(), wb.cuda())
+    sa.debug_set(sa.DEBUG_GATE_WIDE_TILES, 1 if wide else 0)
+    try:
+        launches = sa.launch_count()
+        if dual:
+            out = sa.sa_gate_projection_forward(ya.cuda(), wa.cuda(), yb.cuda(), wb.cuda())
+        else:
+            out = sa.sa_gate_projection_forward(ya.cuda(), wa.cuda())
+        # the two kernels differ in their launch count on the dual path (one per path / one)
+        if dual:
+            assert sa.launch_count() - launches == (2 if wide else 1)
+    finally:
+        sa.debug_set(sa.DEBUG_GATE_WIDE_TILES, 1)
     assert sa.sa_read_status() == 0
-    idx = torch.tensor([0, 1, 127, 128, 2047, 4095])
-    _check(out[idx.cuda()], ya[idx], wa, yb[idx], wb, dm, 2e-2)
+    idx = _model_width_rows(rows, np.random.default_rng(3))
+    _check(out[idx.cuda()], ya[idx], wa, yb[idx] if dual else None, wb if dual else None, dm, 2e-2)
 
 
 def test_rejects_bad_arguments():

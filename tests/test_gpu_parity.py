@@ -95,8 +95,7 @@ def test_sa_forward_small(B, Hq, Hkv, n, d, w, flags, dtype):
     assert sa.sa_read_status() == 0
 
 
-@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
-@pytest.mark.parametrize("B,Hq,Hkv,n,d,w,flags", [
+SWA_SMALL = [
     (2, 4, 2, 300, 64, 33, CAUSAL | SWA_ONE_SIDED),
     (1, 2, 1, 257, 128, 64, CAUSAL | SWA_ONE_SIDED),
     (1, 2, 2, 96, 128, 500, CAUSAL | SWA_ONE_SIDED),
@@ -104,7 +103,11 @@ def test_sa_forward_small(B, Hq, Hkv, n, d, w, flags, dtype):
     (2, 4, 2, 300, 64, 33, CAUSAL),
     (2, 4, 2, 300, 64, 33, 0),
     (1, 1, 1, 200, 128, 31, LINEAR_WINDOW),
-])
+]
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("B,Hq,Hkv,n,d,w,flags", SWA_SMALL)
 def test_swa_forward_small(B, Hq, Hkv, n, d, w, flags, dtype):
     q, k, v = draw((B, Hq, n, d), (B, Hkv, n, d), dtype, seed=3 * n + w)
     y, lse = sa.sa_swa_forward(q.cuda(), k.cuda(), v.cuda(), w, flags, want_lse=True)
@@ -113,29 +116,60 @@ def test_swa_forward_small(B, Hq, Hkv, n, d, w, flags, dtype):
     assert np.abs(as_f64(lse) - rlse).max() <= (1e-4 if dtype == torch.float32 else 2e-2)
 
 
-@pytest.mark.parametrize("block", ["64", "128"])
-def test_both_score_block_widths(block):
-    # the tensor-core forward has a 64-key and a 128-key score block; the library picks by w,
-    # a child process with SA_KEY_BLOCK set runs the other one on the same cases
-    import os, subprocess, sys
-    env = dict(os.environ, SA_KEY_BLOCK=block)
-    r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-m", "gpu", __file__, "-k",
-                        "test_sa_forward_small or test_swa_forward_small or test_gated_forward_small or "
-                        "test_backward_small"],
-                       env=env, capture_output=True, text=True)
-    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+@pytest.fixture
+def debug_option():
+    """Sets a test hook of the library for one test and restores the default afterwards."""
+    defaults = {sa.DEBUG_SCORE_BLOCK: 0, sa.DEBUG_SWA_TILE_LOADS: 1, sa.DEBUG_TENSOR_CORES: 1,
+                sa.DEBUG_GATE_WIDE_TILES: 1}
+    touched = []
+
+    def set_(key, value):
+        touched.append(key)
+        sa.debug_set(key, value)
+    yield set_
+    for key in touched:
+        sa.debug_set(key, defaults[key])
 
 
-def test_swa_branch_without_tma_tile_loads():
+@pytest.mark.parametrize("block", [64, 128])
+def test_both_score_block_widths(block, debug_option):
+    # the tensor-core kernels have a 64-key and a 128-key score block; the library picks by w,
+    # the test hook forces each in turn on the same cases (bf16 only: fp32 never runs them)
+    debug_option(sa.DEBUG_SCORE_BLOCK, block)
+    bf = torch.bfloat16
+    for case in SMALL:
+        test_sa_forward_small(*case, bf)
+    for case in SWA_SMALL:
+        test_swa_forward_small(*case, bf)
+    for save in (False, True):
+        test_gated_forward_small(bf, save)
+    for case in BWD_SMALL:
+        for gated in (False, True):
+            test_backward_small(*case, gated, bf)
+
+
+def test_swa_branch_without_tma_tile_loads(debug_option):
     # the one-sided SWA branch loads whole tiles by TMA when its tensors are plain row
-    # matrices; a child process with SA_SWA_TMA=0 runs the cp.async gather on the same cases
-    import os, subprocess, sys
-    env = dict(os.environ, SA_SWA_TMA="0")
-    r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-m", "gpu", __file__, "-k",
-                        "test_swa_forward_small or test_gated_forward_small or "
-                        "test_gated_forward_both_combine_paths"],
-                       env=env, capture_output=True, text=True)
-    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+    # matrices; with the hook off it gathers rows with cp.async like the SA branch
+    debug_option(sa.DEBUG_SWA_TILE_LOADS, 0)
+    bf = torch.bfloat16
+    for case in SWA_SMALL:
+        test_swa_forward_small(*case, bf)
+    for save in (False, True):
+        test_gated_forward_small(bf, save)
+    for fused in (False, True):
+        for token_major in (False, True):
+            test_gated_forward_both_combine_paths(bf, fused, token_major)
+
+
+def test_cuda_core_kernels_on_tensor_core_shapes(debug_option):
+    # with the tensor cores switched off the general kernels serve the bf16 d = 64 / 128 cases
+    debug_option(sa.DEBUG_TENSOR_CORES, 0)
+    bf = torch.bfloat16
+    for case in SMALL[:9]:
+        test_sa_forward_small(*case, bf)
+    for case in BWD_SMALL[:4]:
+        test_backward_small(*case, True, bf)
 
 
 def test_swa_tma_path_ragged_tail_and_strides():
@@ -153,7 +187,72 @@ def test_swa_tma_path_ragged_tail_and_strides():
                 dev = [t.cuda() for t in (q, k, v)]
             y = sa.sa_swa_forward(dev[0], dev[1], dev[2], w, flags, y=torch.empty_like(dev[0]))
             close(y, ry, torch.bfloat16, "d=%d token_major=%s" % (d, token_major))
+        # views of longer buffers whose tails hold NaN (an unwritten KV-cache tail, say): the
+        # last tile must read zeros past token n - 1, not those rows (0 * NaN would poison
+        # every valid query of the tile through P V)
+        pad = 700
+        dev = []
+        for t in (q, k, v):
+            buf = torch.full((B, t.shape[1], pad, d), float("nan"), dtype=torch.bfloat16,
+                             device="cuda")
+            buf[:, :, :n] = t.cuda()
+            dev.append(buf[:, :, :n])
+        assert not dev[0].is_contiguous()
+        ybuf = torch.zeros((B, Hq, pad, d), dtype=torch.bfloat16, device="cuda")
+        y = sa.sa_swa_forward(dev[0], dev[1], dev[2], w, flags, y=ybuf[:, :, :n])
+        assert torch.isfinite(y.float()).all()
+        close(y, ry, torch.bfloat16, "d=%d NaN tail" % d)
     assert sa.sa_read_status() == 0
+
+
+def crafted_perms(n, rng):
+    """Permutations that stress the masked online softmax: (a) slots hold the tokens in
+    decreasing order, so the first half of every query's band is masked out entirely and the
+    running maximum stays at minus infinity for whole score blocks; (b) a random permutation
+    with token 0 moved to the last slot, whose only visible key (itself) is then the last
+    element of the last block of its band under the linear window."""
+    rev = np.arange(n - 1, -1, -1, dtype=np.int32)
+    rnd = rng.permutation(n).astype(np.int32)
+    at0 = int(np.nonzero(rnd == 0)[0][0])
+    rnd[at0], rnd[n - 1] = rnd[n - 1], rnd[at0]
+    out = []
+    for pm in (rev, rnd):
+        iv = np.empty_like(pm)
+        iv[pm] = np.arange(n, dtype=np.int32)
+        out.append((pm[None].copy(), iv[None].copy()))
+    return out
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("n,d,w,flags", [
+    (700, 128, 300, CAUSAL | LINEAR_WINDOW),    # 128-key score blocks, ragged tail
+    (700, 128, 300, CAUSAL),                    # the same with the circular window
+    (900, 64, 100, CAUSAL | LINEAR_WINDOW),     # 64-key score blocks
+    (515, 128, 2000, CAUSAL),                   # window covers the sequence
+])
+def test_forward_large_scores_and_late_first_visible_key(n, d, w, flags, dtype):
+    """Scaled scores of magnitude ~50 (Q, K ~ 4 N(0,1)), so that exp2 arguments span far more
+    than the lazy-rescaling threshold and a missed rescale or a stale maximum would overflow
+    or flush a row to zero; on permutations whose rows meet their first visible key late."""
+    B, Hq, Hkv = 1, 2, 1
+    q, k, v = draw((B, Hq, n, d), (B, Hkv, n, d), dtype, seed=n + d, scale=1.0)
+    q, k = (q.float() * 4).to(dtype), (k.float() * 4).to(dtype)
+    s_abs = (as_f64(q)[0, 0] @ as_f64(k)[0, 0].T / np.sqrt(d))
+    assert np.abs(s_abs).max() > 40
+    for permc, invc in crafted_perms(n, np.random.default_rng(n)):
+        perm, inv = torch.from_numpy(permc).cuda(), torch.from_numpy(invc).cuda()
+        y, lse = sa.sa_forward(q.cuda(), k.cuda(), v.cuda(), perm, inv, w, flags, want_lse=True)
+        assert sa.sa_read_status() == 0
+        assert torch.isfinite(y.float()).all() and torch.isfinite(lse).all()
+        ry, rlse = oracle.sa_forward(as_f64(q), as_f64(k), as_f64(v), permc, invc, w, flags)
+        close(y, ry, dtype, "y")
+        # lse is of the order of the largest score here: compare relative to its size
+        tol = (1e-4 if dtype == torch.float32 else 2e-2) * max(1.0, np.abs(rlse).max() / 8)
+        assert np.abs(as_f64(lse) - rlse).max() <= tol
+    # the plain-SWA kernels on the same scores (one-sided window: first blocks fully visible)
+    y = sa.sa_swa_forward(q.cuda(), k.cuda(), v.cuda(), w, CAUSAL | SWA_ONE_SIDED)
+    ry, _ = oracle.swa_forward(as_f64(q), as_f64(k), as_f64(v), w, CAUSAL | SWA_ONE_SIDED)
+    close(y, ry, dtype, "y_swa")
 
 
 def test_identity_permutation_equals_swa_on_device():
@@ -339,9 +438,7 @@ def run_backward(q, k, v, dy, lg, perm, inv, w, flags):
                           flags)
 
 
-@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
-@pytest.mark.parametrize("gated", [False, True])
-@pytest.mark.parametrize("B,Hq,Hkv,n,d,w,flags", [
+BWD_SMALL = [
     (2, 4, 2, 200, 64, 21, CAUSAL | SWA_ONE_SIDED),
     (1, 2, 2, 130, 128, 40, 0),
     (1, 2, 1, 77, 32, 300, CAUSAL),
@@ -350,7 +447,12 @@ def run_backward(q, k, v, dy, lg, perm, inv, w, flags):
     (2, 2, 1, 515, 64, 129, CAUSAL | LINEAR_WINDOW),    # no wrap, ragged last tile
     (1, 2, 2, 384, 128, 96, 0),                         # non-causal, n a tile multiple
     (1, 2, 1, 200, 64, 1000, CAUSAL | SWA_ONE_SIDED),   # w > n: every causal key, two tiles
-])
+]
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("gated", [False, True])
+@pytest.mark.parametrize("B,Hq,Hkv,n,d,w,flags", BWD_SMALL)
 def test_backward_small(B, Hq, Hkv, n, d, w, flags, gated, dtype):
     q, k, v = draw((B, Hq, n, d), (B, Hkv, n, d), dtype, seed=n)
     g = torch.Generator().manual_seed(n + 1)
@@ -493,6 +595,31 @@ def test_coverage_study_sa_against_swa_and_prop2_bound():
 
 
 # ----------------------------------------------------------------------- status
+
+def test_bounded_wait_runs_out_and_reports_timeout():
+    """The failure path of the kernels' bounded waits, provoked without breaking anything: a
+    hook kernel waits with the library's wait routine on a barrier nothing completes, with a
+    limit of about a millisecond; it must return on its own, the status word must read
+    SA_ERR_TIMEOUT (6), tensor-core launches are skipped while it is set, and reading clears
+    it so that the next call works again."""
+    B, Hq, Hkv, n, d, w = 1, 2, 1, 300, 64, 40
+    q, k, v = draw((B, Hq, n, d), (B, Hkv, n, d), torch.bfloat16, seed=12)
+    perm, inv, _, _ = perms(12, 0, B, n)
+    qd, kd, vd = q.cuda(), k.cuda(), v.cuda()
+    good = sa.sa_forward(qd, kd, vd, perm, inv, w, CAUSAL)
+    assert sa.sa_read_status() == 0
+    sa.debug_wait_timeout(2_000_000)
+    torch.cuda.synchronize()                       # the kernel came back by itself
+    sentinel = torch.full_like(good, 7.0)
+    sa.sa_forward(qd, kd, vd, perm, inv, w, CAUSAL, y=sentinel)   # skipped: status is sticky
+    assert sa.sa_read_status() == 6
+    assert torch.equal(sentinel, torch.full_like(good, 7.0))
+    assert sa.sa_read_status() == 0                # reading cleared it
+    again = sa.sa_forward(qd, kd, vd, perm, inv, w, CAUSAL)
+    assert sa.sa_read_status() == 0 and torch.equal(again, good)
+    with pytest.raises(sa.SaError):
+        sa.debug_wait_timeout(0)
+
 
 def test_validate_perm_reports_a_non_bijection():
     B, Hq, Hkv, n, d, w = 1, 1, 1, 64, 64, 9

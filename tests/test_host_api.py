@@ -95,3 +95,34 @@ def test_status_strings():
     assert sa.status_string(0) == "ok"
     assert "workspace" in sa.status_string(3)
     assert "permutation" in sa.status_string(5)
+
+
+def test_debug_hooks_validate_their_arguments():
+    lib = sa.load_library()
+    assert lib.sa_debug_set(99, 0) == 1
+    assert lib.sa_debug_set(sa.DEBUG_SCORE_BLOCK, 96) == 1
+    assert lib.sa_debug_set(sa.DEBUG_TENSOR_CORES, 2) == 1
+    for key, default in ((sa.DEBUG_SCORE_BLOCK, 0), (sa.DEBUG_SWA_TILE_LOADS, 1),
+                         (sa.DEBUG_TENSOR_CORES, 1), (sa.DEBUG_GATE_WIDE_TILES, 1)):
+        assert lib.sa_debug_set(key, default) == 0
+    assert lib.sa_debug_wait_timeout(0, None) == 1          # rejected before any launch
+    assert lib.sa_debug_wait_timeout(1 << 40, None) == 1
+
+
+def test_library_reads_no_environment_variable():
+    # kernel choice must not depend on the environment: no getenv in the sources
+    csrc = os.path.join(ROOT, "paper_2604_00754_b200", "csrc")
+    for name in os.listdir(csrc):
+        assert "getenv" not in open(os.path.join(csrc, name)).read(), name
+
+
+def test_stale_library_is_not_loaded_when_the_rebuild_fails(tmp_path, monkeypatch):
+    from paper_2604_00754_b200 import build as b
+    monkeypatch.setattr(sa, "_lib", None)
+    monkeypatch.setattr(b, "stale", lambda: True)
+
+    def fail(*a, **k):
+        raise OSError("no compiler")
+    monkeypatch.setattr(b, "build_library", fail)
+    with pytest.raises(RuntimeError, match="older than its sources"):
+        sa.load_library()
