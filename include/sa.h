@@ -161,6 +161,35 @@ sa_status sa_swa_gated_forward(const sa_problem* p, const void* q, const void* k
                                float* lse_sa, float* lse_swa, void* ws, size_t ws_bytes,
                                sa_stream_t stream);
 
+/* sa_make_perm + sa_swa_gated_forward (Alg. 1 line 1, Alg. 2, Eq. 5) for tensors that live in
+ * HOST memory: q, k, v, y are host pointers to contiguous [B,H,n,d] tensors of p->dtype
+ * (p's stride fields are ignored), gate_logits a host pointer to fp32 [2,Hq]; pinned memory
+ * lets the copies overlap the kernels, pageable memory works but serialises.  The KV heads
+ * travel through the GPU in n_groups contiguous ranges (a range of one KV head in q_parts
+ * ranges of its query heads when they divide evenly), on three internal streams: copy in,
+ * compute, copy out.  The permutation is drawn from (seed, layer) as in sa_make_perm and
+ * shared by all ranges; the gates are applied by the streaming combine of
+ * sa_swa_gated_forward, so the result has the bits of that call given scratch.
+ *   ws: DEVICE workspace of sa_host_forward_ws_bytes(p) bytes, 256-byte aligned, owned by the
+ *       caller (device copies of q, k, v, y, one branch output, the permutation and its
+ *       scratch).  No device memory is allocated; the first call on a device creates the
+ *       three streams and the events of the pipeline and keeps them.
+ *   stream: the call is ordered after what `stream` has queued, and `stream` waits for the
+ *       last copy out, so the caller synchronises (or times) on `stream` alone.  y must not
+ *       be read on the host before that.  Calls on one device must not overlap.
+ * Errors: SA_ERR_INVALID_ARG, SA_ERR_WORKSPACE, SA_ERR_CUDA, and those of the two calls. */
+size_t sa_host_forward_ws_bytes(const sa_problem* p);
+sa_status sa_swa_gated_forward_host(const sa_problem* p, const void* q, const void* k,
+                                    const void* v, const float* gate_logits, void* y,
+                                    uint64_t seed, uint32_t layer, int32_t n_groups,
+                                    int32_t q_parts, void* ws, size_t ws_bytes,
+                                    sa_stream_t stream);
+/* The head ranges sa_swa_gated_forward_host uses, for inspection (host only, no GPU needed):
+ * writes up to max_pieces rows of (kv_begin, kv_end, q_begin, q_end, carries_kv) and returns
+ * their number, or -1 for bad head counts or too small an array. */
+int32_t sa_host_forward_plan(int32_t Hq, int32_t Hkv, int32_t n_groups, int32_t q_parts,
+                             int32_t* pieces, int32_t max_pieces);
+
 /* Backward of sa_forward (gate_logits == NULL: y_swa, lse_swa, dgate_logits ignored, y_sa
  * is the forward's y) or of sa_swa_gated_forward.  The paper only times this pass
  * (Sec. 4.3); the formulas are the derivative of Eq. 1 / Eq. 5 with sigma constant:

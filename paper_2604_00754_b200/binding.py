@@ -30,6 +30,7 @@ EXPORTS = [
     "sa_status_string", "sa_launch_count", "sa_set_profile_events", "sa_make_perm_static",
     "sa_gate_projection_forward", "sa_gate_projection_backward",
     "sa_gate_projection_backward_ws_bytes", "sa_debug_set", "sa_debug_wait_timeout",
+    "sa_swa_gated_forward_host", "sa_host_forward_ws_bytes", "sa_host_forward_plan",
 ]
 DEBUG_SCORE_BLOCK, DEBUG_SWA_TILE_LOADS, DEBUG_TENSOR_CORES, DEBUG_GATE_WIDE_TILES = range(4)
 
@@ -103,6 +104,12 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.sa_set_profile_events.restype = None
     lib.sa_launch_count.argtypes = []
     lib.sa_launch_count.restype = u64
+    lib.sa_host_forward_ws_bytes.argtypes = [pp]
+    lib.sa_host_forward_ws_bytes.restype = sz
+    lib.sa_host_forward_plan.argtypes = [i32, i32, i32, i32, vp, i32]
+    lib.sa_host_forward_plan.restype = i32
+    lib.sa_swa_gated_forward_host.argtypes = [pp, vp, vp, vp, vp, vp, u64, u32, i32, i32, vp, sz, vp]
+    lib.sa_swa_gated_forward_host.restype = ctypes.c_int
     lib.sa_debug_set.argtypes = [ctypes.c_int, ctypes.c_int]
     lib.sa_debug_set.restype = ctypes.c_int
     lib.sa_debug_wait_timeout.argtypes = [i64, vp]
@@ -399,6 +406,42 @@ def sa_gate_projection_backward(dout, y_sa, w_sa, y_swa=None, w_swa=None, ws=Non
         _ptr(w_sa), _ptr(w_swa), _ptr(dy_sa), _ptr(dy_swa), dy_sa.stride(0), _ptr(dw_sa),
         _ptr(dw_swa), _ptr(ws), ws.numel(), _stream()), "sa_gate_projection_backward")
     return (dy_sa, dw_sa, dy_swa, dw_swa) if dual else (dy_sa, dw_sa)
+
+
+def host_forward_plan(Hq: int, Hkv: int, n_groups: int, q_parts: int):
+    """Head ranges of the host-memory forward: (kv_begin, kv_end, q_begin, q_end, carries_kv)."""
+    buf = (ctypes.c_int32 * (5 * 256))()
+    cnt = int(load_library().sa_host_forward_plan(Hq, Hkv, n_groups, q_parts, buf, 256))
+    if cnt < 0:
+        raise ValueError("Hq must be a positive multiple of Hkv")
+    return [tuple(buf[5 * i + j] for j in range(4)) + (bool(buf[5 * i + 4]),) for i in range(cnt)]
+
+
+def host_forward_ws_bytes(B, Hq, Hkv, n, d, dtype=BF16) -> int:
+    p = SaProblem(B=B, Hq=Hq, Hkv=Hkv, n=n, d=d, w=1, dtype=dtype)
+    r = int(load_library().sa_host_forward_ws_bytes(ctypes.byref(p)))
+    if r == ctypes.c_size_t(-1).value:
+        raise SaError(1, "sa_host_forward_ws_bytes")
+    return r
+
+
+def sa_swa_gated_forward_host(q, k, v, gate_logits, y, w, flags, seed, layer, ws, n_groups=8,
+                              q_parts=2, scale=0.0):
+    """Fresh permutation + gated SA+SWA forward on HOST tensors (contiguous [B,H,n,d], pinned
+    for overlap); ws: CUDA uint8 tensor of host_forward_ws_bytes(...).  y (host) is complete
+    once the current stream has been synchronised."""
+    for t in (q, k, v, y, gate_logits):
+        if t.is_cuda or not t.is_contiguous():
+            raise ValueError("host tensors must be contiguous CPU tensors")
+    dt = {torch.float32: F32, torch.bfloat16: BF16}[q.dtype]
+    B, Hq, n, d = q.shape
+    p = SaProblem(B=B, Hq=Hq, Hkv=k.shape[1], n=n, d=d, w=int(w), dtype=dt, flags=int(flags),
+                  softmax_scale=float(scale))
+    _check(load_library().sa_swa_gated_forward_host(
+        ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(gate_logits), _ptr(y),
+        int(seed) & (2 ** 64 - 1), int(layer), int(n_groups), int(q_parts), _ptr(ws), ws.numel(),
+        _stream()), "sa_swa_gated_forward_host")
+    return y
 
 
 def sa_read_status() -> int:

@@ -3,38 +3,53 @@ the bits of the single device-resident call."""
 import pytest
 import torch
 
+from paper_2604_00754_b200 import binding as sab
 from paper_2604_00754_b200 import host
 
 
 def test_head_groups_cover_every_head_once():
     for Hq, Hkv, ng in [(32, 8, 8), (32, 8, 3), (12, 12, 5), (4, 1, 8), (16, 4, 1)]:
-        groups = host.head_groups(Hq, Hkv, ng)
+        groups = sab.host_forward_plan(Hq, Hkv, ng, 1)
         assert len(groups) <= max(1, min(ng, Hkv))
         G = Hq // Hkv
         kv_seen, q_seen = [], []
-        for ka, kb, qa, qb in groups:
-            assert kb > ka and (qa, qb) == (ka * G, kb * G)
+        for ka, kb, qa, qb, with_kv in groups:
+            assert kb > ka and (qa, qb) == (ka * G, kb * G) and with_kv
             kv_seen += list(range(ka, kb))
             q_seen += list(range(qa, qb))
         assert kv_seen == list(range(Hkv)) and q_seen == list(range(Hq))
 
 
 def test_split_query_heads_keeps_coverage_and_kv_ownership():
-    g = host.split_query_heads(host.head_groups(32, 8, 8), 2)
+    g = sab.host_forward_plan(32, 8, 8, 2)
     assert len(g) == 16
     assert [x[2:4] for x in g] == [(2 * i, 2 * i + 2) for i in range(16)]
     assert [x[4] for x in g] == [True, False] * 8          # K/V travel with the first part only
     assert all(kb - ka == 1 for ka, kb, *_ in g)
     # ranges with several KV heads, or an odd number of query heads per KV head, stay whole
-    assert host.split_query_heads(host.head_groups(8, 4, 2), 2) == [(0, 2, 0, 4, True), (2, 4, 4, 8, True)]
-    assert host.split_query_heads(host.head_groups(3, 1, 1), 2) == [(0, 1, 0, 3, True)]
+    assert sab.host_forward_plan(8, 4, 2, 2) == [(0, 2, 0, 4, True), (2, 4, 4, 8, True)]
+    assert sab.host_forward_plan(3, 1, 1, 2) == [(0, 1, 0, 3, True)]
 
 
 def test_head_groups_rejects_bad_head_counts():
     with pytest.raises(ValueError):
-        host.head_groups(10, 4, 2)
+        sab.host_forward_plan(10, 4, 2, 1)
     with pytest.raises(ValueError):
-        host.head_groups(0, 1, 1)
+        sab.host_forward_plan(0, 1, 1, 1)
+
+
+def test_host_forward_rejects_bad_arguments_before_any_cuda_call():
+    import ctypes
+    lib = sab.load_library()
+    p = sab.SaProblem(B=1, Hq=4, Hkv=2, n=64, d=64, w=8, dtype=sab.BF16, flags=sab.CAUSAL)
+    need = sab.host_forward_ws_bytes(1, 4, 2, 64, 64)
+    assert need >= (3 * 4 + 2 * 2) * 64 * 64 * 2       # q, y, scratch + k, v
+    fake = ctypes.c_void_p(0x10000)
+    args = lambda ws, nbytes: (ctypes.byref(p), fake, fake, fake, fake, fake, 1, 0, 2, 1, ws,
+                               nbytes, None)
+    assert lib.sa_swa_gated_forward_host(*args(None, need)) == 1
+    assert lib.sa_swa_gated_forward_host(*args(ctypes.c_void_p(0x10010), need)) == 1   # alignment
+    assert lib.sa_swa_gated_forward_host(*args(fake, need - 1)) == 3
 
 
 @pytest.mark.gpu
