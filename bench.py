@@ -179,9 +179,11 @@ def main():
     ap.add_argument("--workload", default="C3")
     ap.add_argument("--n", type=int, default=0,
                     help="override the sequence length (profiling captures on a smaller case)")
-    ap.add_argument("--leg", default="step", choices=["step", "backward"],
-                    help="backward: time the gated backward of the workload instead of the step "
-                         "(a side measurement with its own JSON line; used for profiling)")
+    ap.add_argument("--leg", default="step",
+                    choices=["step", "backward", "sa_fwd", "swa_fwd", "coverage"],
+                    help="side measurements with their own JSON line (used for profiling): "
+                         "backward = gated backward of the workload; sa_fwd / swa_fwd = that "
+                         "branch's forward alone; coverage = the reach study of Prop. 2")
     ap.add_argument("--no-extras", action="store_true",
                     help="skip the side measurements (SWA, backward, e2e, CPU oracle)")
     args = ap.parse_args()
@@ -228,6 +230,13 @@ def main():
 
     if args.leg == "backward":
         backward_leg(args, c, sa, torch, dev, perm, inv, ws, rank)
+        return
+    if args.leg in ("sa_fwd", "swa_fwd"):
+        branch_leg(args, c, sa, torch, dev, perm, inv, ws, y, pk, rank)
+        return
+    if args.leg == "coverage":
+        if rank == 0:
+            print(json.dumps({"leg": "coverage", "coverage_study": coverage_study(sa, torch, wl)}))
         return
 
     layer = [0]
@@ -338,6 +347,66 @@ def backward_leg(args, c, sa, torch, dev, perm, inv, ws, rank):
                           "config": workload_config(c), "dtype": "bf16", "data": "synthetic"}))
 
 
+def branch_leg(args, c, sa, torch, dev, perm, inv, ws, y, pk, rank):
+    """One branch's forward alone (the kernel the roofline entry is about, or its SWA twin)."""
+    q, k, v = dev["q"], dev["k"], dev["v"]
+    sa.sa_make_perm(c.seed, 0, c.B, c.n, perm=perm, inv=inv, ws=ws)
+    if args.leg == "sa_fwd":
+        fn = lambda: sa.sa_forward(q, k, v, perm, inv, c.w, c.flags, y=y)
+    else:
+        fn = lambda: sa.sa_swa_forward(q, k, v, c.w, c.flags, y=y)
+    ms = event_ms(fn, args.steps, args.warmup, torch)
+    assert sa.sa_read_status() == 0
+    tf = 4.0 * c.B * c.Hq * c.n * c.w * c.d / (ms * 1e-3) / 1e12
+    if rank == 0:
+        print(json.dumps({"leg": args.leg, "ms": ms, "tokens_per_s": c.B * c.n / (ms * 1e-3),
+                          "tflops_nominal": tf, "frac_of_burst": tf / pk["bf16_tflops"],
+                          "steps": args.steps, "warmup": args.warmup,
+                          "config": workload_config(c), "dtype": "bf16", "data": "synthetic"}))
+
+
+def coverage_study(sa, torch, wl):
+    """Fig. 2 (left) / Prop. 2 as numbers: seed-averaged |R_l| through sa_coverage for SA with an
+    independent permutation per layer (the paper's default), SA with one fixed permutation reused
+    at every layer (Sec. 3.3 deterministic mode), and plain SWA, beside Prop. 2's expansion
+    bound applied to the measured mean; at the paper's n = 2048, w = 32 and at the (n, w) of the
+    pre-training and the two Qwen3-shaped workloads.  Non-causal mask, as in the proposition."""
+    import numpy as np
+    out = {}
+    cases = [("fig2_n2048_w32", 2048, 32, 6, 16), ("C5_n4096_w128", 4096, 128, 4, 8),
+             ("C3_n32768_w1024", 32768, 1024, 3, 4), ("C4_n131072_w2048", 131072, 2048, 3, 2)]
+    for name, n, w, L, seeds in cases:
+        h = (w + 1) // 2 - 1
+        band = min(n, 2 * h + 1)
+        pr = (band - 1) / (n - 1)
+        src = n // 3
+        indep = np.zeros((seeds, L))
+        fixed = np.zeros((seeds, L))
+        t0 = time.perf_counter()
+        for s_ in range(seeds):
+            pl = [sa.sa_make_perm(9000 + s_, l, 1, n) for l in range(L)]
+            perm = torch.cat([a for a, _ in pl]).contiguous()
+            inv = torch.cat([b for _, b in pl]).contiguous()
+            indep[s_] = sa.sa_coverage(perm, inv, w, 0, src, want_row_count=False)[2].cpu().numpy()
+            p1 = pl[0][0].repeat(L, 1).contiguous()
+            i1 = pl[0][1].repeat(L, 1).contiguous()
+            fixed[s_] = sa.sa_coverage(p1, i1, w, 0, src, want_row_count=False)[2].cpu().numpy()
+        ident = torch.arange(n, dtype=torch.int32, device="cuda").repeat(L, 1).contiguous()
+        swa = sa.sa_coverage(ident, ident, w, 0, src, want_row_count=False)[2].cpu().numpy()
+        torch.cuda.synchronize()
+        mean = indep.mean(axis=0)
+        bound = [float(band)] + [float((r + (n - r) * (1 - (1 - pr) ** r)).mean())
+                                 for r in indep[:, :-1].T]
+        out[name] = {"n": n, "w": w, "band": band, "layers": L, "seeds": seeds,
+                     "sa_independent_sigma_mean_reach": [float(x) for x in mean],
+                     "prop2_lower_bound_on_mean": bound,
+                     "sa_fixed_sigma_mean_reach": [float(x) for x in fixed.mean(axis=0)],
+                     "swa_reach": [int(x) for x in swa],
+                     "swa_closed_form": [min(n, 2 * (l + 1) * h + 1) for l in range(L)],
+                     "seconds": time.perf_counter() - t0}
+    return out
+
+
 def extras(args, c, wl, sa, torch, dev, host, perm, inv, ws, y, pk):
     """Side measurements on rank 0, outside the timed region of `value`."""
     q, k, v, lg = dev["q"], dev["k"], dev["v"], dev["gate_logits"]
@@ -360,22 +429,107 @@ def extras(args, c, wl, sa, torch, dev, host, perm, inv, ws, y, pk):
     res["sa_overhead_vs_swa"] = sa_ms / swa_ms - 1.0
     res["make_perm_ms"] = perm_ms
 
-    # end to end through the host-memory API: pinned host inputs -> device, fresh permutation,
-    # gated forward, result back to pinned host memory; the KV-head groups are pipelined so
-    # that copies in, kernels and copies out overlap
-    from paper_2604_00754_b200 import host as sa_host
+    # end to end through the C entry point that takes HOST buffers: pinned host inputs ->
+    # device, fresh permutation, gated forward, result back to pinned host memory, all inside
+    # the timed region; the library pipelines the KV-head groups on three streams so that
+    # copies in, kernels and copies out overlap
     hy = torch.empty_like(host["q"]).pin_memory()
-    hf = sa_host.HostForward(c.B, c.Hq, c.Hkv, c.n, c.d, c.w, c.flags, n_groups=8)
+    hg = host["gate_logits"].pin_memory()
+    hws = torch.empty(sa.host_forward_ws_bytes(c.B, c.Hq, c.Hkv, c.n, c.d), dtype=torch.uint8,
+                      device="cuda")
     layer = [1000]
 
     def e2e_step():
-        hf.forward(host["q"], host["k"], host["v"], host["gate_logits"], hy, c.seed, layer[0])
+        sa.sa_swa_gated_forward_host(host["q"], host["k"], host["v"], hg, hy, c.w, c.flags,
+                                     c.seed, layer[0], hws, n_groups=8, q_parts=2)
         layer[0] += 1
     e2e_ms = event_ms(e2e_step, it, 2, torch)
+    elt = host["q"].element_size()
     res["e2e"] = {"value": c.B * c.n / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms,
-                  "h2d_bytes_per_step": hf.h2d_bytes(), "d2h_bytes_per_step": hf.d2h_bytes(),
-                  "api": "host.HostForward.forward, 8 KV-head groups x 2 query-head parts on 3 streams"}
-    del hf
+                  "h2d_bytes_per_step": sum(host[x].numel() for x in ("q", "k", "v")) * elt
+                                        + hg.numel() * 4,
+                  "d2h_bytes_per_step": hy.numel() * elt,
+                  "api": "sa_swa_gated_forward_host (C ABI, host pointers), 8 KV-head groups x 2 "
+                         "query-head parts on 3 streams"}
+    del hws
+    torch.cuda.empty_cache()
+
+    # gated backward at the same workload (forward once, saving what the backward needs)
+    if c.n * c.Hq <= 32768 * 32:
+        dyb = torch.randn(q.shape, generator=torch.Generator(device="cuda").manual_seed(c.seed + 77),
+                          device="cuda", dtype=torch.float32).to(q.dtype)
+        sv = sa.sa_swa_gated_forward(q, k, v, perm, inv, lg, c.w, c.flags, save_for_bwd=True)
+        bws3 = torch.empty(sa.sa_workspace_bytes(sa.make_problem(q, k, c.w, c.flags), sa.OP_BACKWARD),
+                           dtype=torch.uint8, device="cuda")
+        bo = {}
+
+        def bwd_main():
+            r = sa.sa_backward(q, k, v, perm, inv, lg, sv[1], sv[2], sv[3], sv[4], dyb, c.w,
+                               c.flags, ws=bws3, out=bo)
+            bo.update(zip(("dq", "dk", "dv", "dgate"), r))
+        bms = event_ms(bwd_main, max(3, it // 2), 2, torch)
+        bfl = 2 * 2.5 * flops
+        res["backward_%s" % c.name.split("_")[0]] = {
+            "gated_bwd_ms": bms, "tokens_per_s": c.B * c.n / (bms * 1e-3),
+            "tflops_nominal": bfl / (bms * 1e-3) / 1e12,
+            "frac_of_burst": bfl / (bms * 1e-3) / 1e12 / pk["bf16_tflops"]}
+        del dyb, sv, bws3, bo
+        torch.cuda.empty_cache()
+
+    # single-layer SA forward on the HBM-bound shape: tokens/s and the achieved bytes per second
+    # over the algorithmic bytes (Q, K, V in, Y out, each once)
+    c2 = wl.C2
+    t2 = {k_: v_.cuda() for k_, v_ in wl.draw(c2).items()}
+    p2, i2 = sa.sa_make_perm(c2.seed, 0, c2.B, c2.n)
+    # rotate among enough copies of the inputs to exceed L2 (134 MB per copy, L2 126 MB)
+    copies = [{k_: t2[k_].clone() for k_ in ("q", "k", "v")} for _ in range(3)]
+    y2 = torch.empty_like(t2["q"])
+    turn = [0]
+
+    def fwd2():
+        cp = copies[turn[0] % len(copies)]
+        turn[0] += 1
+        sa.sa_forward(cp["q"], cp["k"], cp["v"], p2, i2, c2.w, c2.flags, y=y2)
+    ms2 = event_ms(fwd2, max(20, it), 3, torch)
+    bytes2 = 2.0 * (2 * c2.B * c2.Hq + 2 * c2.B * c2.Hkv) * c2.n * c2.d
+    fl2 = 4.0 * c2.B * c2.Hq * c2.n * c2.w * c2.d
+    res["C2_layer"] = {
+        "sa_fwd_ms": ms2, "tokens_per_s": c2.B * c2.n / (ms2 * 1e-3),
+        "algorithmic_bytes": bytes2, "achieved_gbs": bytes2 / (ms2 * 1e-3) / 1e9,
+        "frac_of_hbm": bytes2 / (ms2 * 1e-3) / 1e9 / pk["hbm_gbs"],
+        "tflops_nominal": fl2 / (ms2 * 1e-3) / 1e12,
+        "l2_policy": "3 input copies in rotation (402 MB > L2)"}
+    del t2, copies, y2
+    torch.cuda.empty_cache()
+
+    # long-context prefill: 48 layers back to back, each a fresh permutation + gated forward
+    c4 = wl.C4
+    t4 = {k_: v_.cuda() for k_, v_ in wl.draw(c4).items()}
+    p4 = torch.empty(c4.B, c4.n, dtype=torch.int32, device="cuda")
+    i4 = torch.empty_like(p4)
+    y4 = torch.empty_like(t4["q"])
+    ws4 = torch.empty(sa.sa_workspace_bytes(sa.SaProblem(B=c4.B, n=c4.n), sa.OP_MAKE_PERM),
+                      dtype=torch.uint8, device="cuda")
+    g4 = torch.empty(sa.sa_workspace_bytes(sa.make_problem(t4["q"], t4["k"], c4.w, c4.flags),
+                                           sa.OP_GATED_FORWARD_SCRATCH), dtype=torch.uint8,
+                     device="cuda")
+
+    def prefill():
+        for l in range(c4.layers):
+            sa.sa_make_perm(c4.seed, l, c4.B, c4.n, perm=p4, inv=i4, ws=ws4)
+            sa.sa_swa_gated_forward(t4["q"], t4["k"], t4["v"], p4, i4, t4["gate_logits"], c4.w,
+                                    c4.flags, out={"y": y4}, ws=g4)
+    ms4 = event_ms(prefill, 2, 1, torch)
+    fl4 = 2 * 4.0 * c4.B * c4.Hq * c4.n * c4.w * c4.d * c4.layers
+    res["C4_prefill_48_layers"] = {
+        "total_ms": ms4, "ms_per_layer": ms4 / c4.layers,
+        "tokens_per_s": c4.B * c4.n / (ms4 * 1e-3),
+        "layer_tokens_per_s": c4.B * c4.n * c4.layers / (ms4 * 1e-3),
+        "tflops_nominal": fl4 / (ms4 * 1e-3) / 1e12,
+        "frac_of_sustained": fl4 / (ms4 * 1e-3) / 1e12 / pk["bf16_tflops_sustained"],
+        "frac_of_burst": fl4 / (ms4 * 1e-3) / 1e12 / pk["bf16_tflops"]}
+    del t4, p4, i4, y4, ws4, g4
+    torch.cuda.empty_cache()
 
     # backward on the pre-training shape (fresh permutation, gated forward saving, backward)
     c5 = wl.C5
@@ -399,9 +553,24 @@ def extras(args, c, wl, sa, torch, dev, host, perm, inv, ws, y, pk):
     f5 = event_ms(fwd5, it, 2, torch)
     b5 = event_ms(bwd5, it, 2, torch)
     fl5 = 2 * 4.0 * c5.B * c5.Hq * c5.n * c5.w * c5.d
+    ws5 = torch.empty(sa.sa_workspace_bytes(sa.SaProblem(B=c5.B, n=c5.n), sa.OP_MAKE_PERM),
+                      dtype=torch.uint8, device="cuda")
+
+    def step5():          # the pre-training step: 12 layers, a fresh permutation each
+        for l in range(c5.layers):
+            sa.sa_make_perm(c5.seed, l, c5.B, c5.n, perm=p5, inv=i5, ws=ws5)
+            fwd5()
+            bwd5()
+    s5 = event_ms(step5, 3, 1, torch)
+    bytes5 = 15 * 2.0 * c5.B * c5.Hq * c5.n * c5.d          # 15 tensor passes of 50.3 MB per layer
     res["pretrain_layer_C5"] = {
         "gated_fwd_ms": f5, "bwd_ms": b5, "tokens_per_s_fwd_bwd": c5.B * c5.n / ((f5 + b5) * 1e-3),
-        "tflops_fwd_bwd": 3.5 * fl5 / ((f5 + b5) * 1e-3) / 1e12}
+        "tflops_fwd_bwd": 3.5 * fl5 / ((f5 + b5) * 1e-3) / 1e12,
+        "step_12_layers_ms": s5, "step_tokens_per_s": c5.B * c5.n / (s5 * 1e-3),
+        "step_tflops_nominal": 3.5 * fl5 * c5.layers / (s5 * 1e-3) / 1e12,
+        "hbm_floor_ms_per_layer": bytes5 / pk["hbm_gbs"] / 1e6,
+        "frac_of_hbm_floor": (bytes5 / pk["hbm_gbs"] / 1e6) / (s5 / c5.layers)}
+    del ws5
     del t5, saved, bout, bws
     torch.cuda.empty_cache()
 
@@ -470,6 +639,8 @@ def extras(args, c, wl, sa, torch, dev, host, perm, inv, ws, y, pk):
         "bwd_dual_frac_of_burst": 6 * gfl / (gb2 * 1e-3) / 1e12 / pk["bf16_tflops"]})
     del ya, yb, wa, wb, og, gbw
     torch.cuda.empty_cache()
+
+    res["coverage_study"] = coverage_study(sa, torch, wl)
 
     rate, dt, rows, threads = oracle_sample_rate(c, host, 196608)
     res["cpu_baseline"] = {

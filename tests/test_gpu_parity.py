@@ -594,6 +594,40 @@ def test_coverage_study_sa_against_swa_and_prop2_bound():
     assert mean[2] > 10 * swa_reach[2].item()       # SA has spread far beyond the local window
 
 
+@pytest.mark.parametrize("n,w,L,seeds", [(2048, 32, 6, 4), (4096, 128, 4, 2), (32768, 1024, 3, 1)])
+def test_coverage_fixed_sigma_against_independent_sigma(n, w, L, seeds):
+    """The paper's two inference modes at the benchmark shapes: one fixed permutation reused at
+    every layer gives the linear growth min(n, 2lh+1) of plain SWA (closed form, any size);
+    an independent permutation per layer respects Prop. 2's expansion bound and covers the
+    sequence within a few layers.  Bit-exact against the oracle where it finishes in seconds."""
+    h = (w + 1) // 2 - 1
+    band = min(n, 2 * h + 1)
+    pr = (band - 1) / (n - 1)
+    src = n // 3
+    for s_ in range(seeds):
+        pl = [sa.sa_make_perm(500 + s_, l, 1, n) for l in range(L)]
+        perm = torch.cat([a for a, _ in pl]).contiguous()
+        inv = torch.cat([b for _, b in pl]).contiguous()
+        nnz, _, reach = sa.sa_coverage(perm, inv, w, 0, src, want_row_count=False)
+        reach = reach.cpu().numpy()
+        assert np.all(nnz.cpu().numpy() == n * band)          # closed form, every permutation
+        assert reach[0] == band and np.all(np.diff(reach) >= 0)
+        # one layer of Prop. 2's bound from the measured set size, with slack for one draw
+        for l in range(L - 1):
+            r = float(reach[l])
+            assert reach[l + 1] >= 0.9 * (r + (n - r) * (1 - (1 - pr) ** r))
+        assert reach[-1] == n
+        fixed_p = pl[0][0].repeat(L, 1).contiguous()
+        fixed_i = pl[0][1].repeat(L, 1).contiguous()
+        _, _, fr = sa.sa_coverage(fixed_p, fixed_i, w, 0, src, want_row_count=False)
+        assert fr.cpu().tolist() == [min(n, 2 * (l + 1) * h + 1) for l in range(L)]
+        if n <= 4096:
+            _, _, oreach = oracle.coverage(perm.cpu().numpy(), inv.cpu().numpy(), w, 0, src)
+            assert np.array_equal(reach, oreach)
+            _, _, ofr = oracle.coverage(fixed_p.cpu().numpy(), fixed_i.cpu().numpy(), w, 0, src)
+            assert np.array_equal(fr.cpu().numpy(), ofr)
+
+
 # ----------------------------------------------------------------------- status
 
 def test_bounded_wait_runs_out_and_reports_timeout():

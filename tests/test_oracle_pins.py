@@ -557,6 +557,26 @@ def test_sa_reach_growth_and_prop2_bound():
     assert mean[3] > 0.99 * n
 
 
+def test_fixed_sigma_reach_is_linear_like_swa():
+    """Deterministic mode (Sec. 3.3: one fixed permutation reused at every layer): in slot
+    space every layer is the same window, so the reachable set is an interval of slots that
+    grows by 2h per layer, min(n, 2lh+1) tokens, exactly as for plain SWA; it is the fresh
+    permutation per layer that gives the fast growth of Prop. 2."""
+    n, w, L = 600, 17, 8
+    h = (w + 1) // 2 - 1
+    perm1, inv1 = oracle.make_perm(77, 0, 1, n)
+    perm = np.repeat(perm1, L, axis=0)
+    inv = np.repeat(inv1, L, axis=0)
+    for src in (0, 250, n - 1):
+        _, _, reach = oracle.coverage(perm, inv, w, 0, src)
+        assert list(reach) == [min(n, 2 * (l + 1) * h + 1) for l in range(L)]
+    # independent permutations from the same source spread much faster
+    pl = [oracle.make_perm(77, l, 1, n) for l in range(L)]
+    _, _, fresh = oracle.coverage(np.concatenate([a for a, _ in pl]),
+                                  np.concatenate([b for _, b in pl]), w, 0, 250)
+    assert fresh[2] > 4 * reach[2] and fresh[3] == n
+
+
 def test_causal_reach_only_moves_backwards():
     n, w, L = 64, 9, 4
     pl = [oracle.make_perm(3, l, 1, n) for l in range(L)]
