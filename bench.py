@@ -184,6 +184,9 @@ def main():
                     help="side measurements with their own JSON line (used for profiling): "
                          "backward = gated backward of the workload; sa_fwd / swa_fwd = that "
                          "branch's forward alone; coverage = the reach study of Prop. 2")
+    ap.add_argument("--score-block", type=int, default=0, choices=[0, 64, 128],
+                    help="force the score-block width of the tensor-core kernels (test hook of "
+                         "the library; 0 = the library's own choice)")
     ap.add_argument("--no-extras", action="store_true",
                     help="skip the side measurements (SWA, backward, e2e, CPU oracle)")
     args = ap.parse_args()
@@ -208,6 +211,8 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     sa.load_library()
+    if args.score_block:
+        sa.debug_set(sa.DEBUG_SCORE_BLOCK, args.score_block)
     pk = peaks()
 
     # Each rank holds its own batch of independent sequences (the path shards over

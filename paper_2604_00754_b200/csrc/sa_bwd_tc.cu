@@ -120,9 +120,6 @@ bwd_tc_kernel(const __grid_constant__ BwdTcParams p) {
   constexpr bool kKeys = MODE == 1;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-  if (cta_should_skip(reinterpret_cast<volatile int*>(smem + C::kOffMisc + 8), p.status,
-                      p.abort_flag))
-    return;
   const uint32_t sbase = smem_u32(smem);
   if (sbase & 1023u) {
     if (threadIdx.x == 0) atomicCAS(p.status, SA_OK, SA_ERR_CUDA);
@@ -146,6 +143,7 @@ bwd_tc_kernel(const __grid_constant__ BwdTcParams p) {
 
   if (threadIdx.x == 0) {
     *gave_up = 0;
+    note_skip(reinterpret_cast<volatile int*>(smem + C::kOffMisc + 8), p.status, p.abort_flag);
     for (int i = 0; i < C::kNumBars; ++i)
       mbar_init(bar(i), (i >= C::kBarPReady && i < C::kBarODone) ? kTile * C::kRowWgs
                         : (i == C::kBarRFull || (i >= C::kBarCFull && i < C::kBarCEmpty))
@@ -161,6 +159,7 @@ bwd_tc_kernel(const __grid_constant__ BwdTcParams p) {
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  SA_LEAVE_IF_SKIPPED(reinterpret_cast<volatile int*>(smem + C::kOffMisc + 8), 0, tmem, kTmemCols)
 
   if (warp >= 1 && warp < 4) {
     // ---------------------------------------------------- gather producers (warps 1-3)

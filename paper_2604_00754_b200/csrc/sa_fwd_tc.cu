@@ -202,9 +202,6 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
   constexpr int kShift = KB == 64 ? 6 : 7;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-  if (cta_should_skip(reinterpret_cast<volatile int*>(smem + C::kOffMisc + 8), p.status,
-                      p.abort_flag))
-    return;
   const uint32_t sbase = smem_u32(smem);
   if (sbase & 1023u) {                        // the swizzled tiles need 1024-byte alignment
     if (threadIdx.x == 0) atomicCAS(p.status, SA_OK, SA_ERR_CUDA);
@@ -217,6 +214,7 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
 
   if (threadIdx.x == 0) {
     *gave_up = 0;
+    note_skip(reinterpret_cast<volatile int*>(smem + C::kOffMisc + 8), p.status, p.abort_flag);
     for (int i = 0; i < C::kNumBars; ++i)
       mbar_init(bar(i), (i >= C::kBarPReady && i < C::kBarPvDone) ? kTile
                         : (i == C::kBarQFull || (i >= C::kBarSlotFull && i < C::kBarSlotEmpty))
@@ -232,6 +230,7 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  SA_LEAVE_IF_SKIPPED(reinterpret_cast<volatile int*>(smem + C::kOffMisc + 8), 0, tmem, kTmemCols)
 
   // Registers move from the producer / issuer warps to the softmax warps, which hold a
   // whole score row each.

@@ -74,8 +74,6 @@ gate_bwd_kernel(const __grid_constant__ BwdGateParams p, const __grid_constant__
   constexpr int kBlock = 2048 / TN;       // column tiles per block of the tile order
   extern __shared__ __align__(1024) uint8_t smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (cta_should_skip(reinterpret_cast<volatile int*>(smem + kOffMisc + 8), p.status, nullptr))
-    return;
   const uint32_t sbase = smem_u32(smem);
   if (sbase & 1023u) {
     if (threadIdx.x == 0) atomicCAS(p.status, SA_OK, SA_ERR_CUDA);
@@ -87,6 +85,7 @@ gate_bwd_kernel(const __grid_constant__ BwdGateParams p, const __grid_constant__
   volatile int* gave_up = reinterpret_cast<volatile int*>(smem + kOffMisc + 4);
   if (threadIdx.x == 0) {
     *gave_up = 0;
+    note_skip(reinterpret_cast<volatile int*>(smem + kOffMisc + 8), p.status, nullptr);
     for (int i = 0; i < kNumBars; ++i) mbar_init(bar(i), (i >= kBarAccEmpty) ? 256 : 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -99,6 +98,7 @@ gate_bwd_kernel(const __grid_constant__ BwdGateParams p, const __grid_constant__
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  SA_LEAVE_IF_SKIPPED(reinterpret_cast<volatile int*>(smem + kOffMisc + 8), 1, tmem, 512u)
   const int total = p.tiles_m * p.tiles_n;
   // blocks of 2048 columns, row tile by row tile inside a block (operand slices stay in L2)
   auto origin = [&](int tile, int* m0, int* n0) {

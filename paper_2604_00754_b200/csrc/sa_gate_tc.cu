@@ -58,8 +58,6 @@ gate_tc_kernel(const __grid_constant__ GateParams p, const __grid_constant__ CUt
                const __grid_constant__ CUtensorMap tm_wswa) {
   extern __shared__ __align__(1024) uint8_t smem[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (cta_should_skip(reinterpret_cast<volatile int*>(smem + kOffMisc + 8), p.status, nullptr))
-    return;
   const uint32_t sbase = smem_u32(smem);
   if (sbase & 1023u) {                        // the swizzled tiles need 1024-byte alignment
     if (threadIdx.x == 0) atomicCAS(p.status, SA_OK, SA_ERR_CUDA);
@@ -72,6 +70,7 @@ gate_tc_kernel(const __grid_constant__ GateParams p, const __grid_constant__ CUt
 
   if (threadIdx.x == 0) {
     *gave_up = 0;
+    note_skip(reinterpret_cast<volatile int*>(smem + kOffMisc + 8), p.status, nullptr);
     for (int i = 0; i < kNumBars; ++i)
       mbar_init(bar(i), (i >= kBarAccEmpty) ? 256 : 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -85,6 +84,7 @@ gate_tc_kernel(const __grid_constant__ GateParams p, const __grid_constant__ CUt
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  SA_LEAVE_IF_SKIPPED(reinterpret_cast<volatile int*>(smem + kOffMisc + 8), 1, tmem, 512u)
   const int total = p.tiles_m * p.tiles_n;
 
   if (warp == 0) {

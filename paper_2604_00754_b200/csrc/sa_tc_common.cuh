@@ -60,19 +60,27 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
 }
 
-// Should this CTA leave before doing anything?  Yes when an earlier check rejected perm/inv
+// Should this CTA leave without doing its work?  Yes when an earlier check rejected perm/inv
 // (abort_flag) or some CTA has already recorded a timeout: the rest of the grid then leaves at
-// once instead of each waiting out its own limit.  Thread 0 reads the words once and the CTA
-// agrees through `slot` (an int in shared memory), so the answer is the same for every thread
-// even if another kernel writes the status word at that moment.  Contains a __syncthreads.
-__device__ __forceinline__ bool cta_should_skip(volatile int* slot, const int* status,
-                                                const int* abort_flag) {
-  if (threadIdx.x == 0)
-    *slot = (abort_flag && *(volatile const int*)abort_flag) ||
-            *(volatile const int*)status == SA_ERR_TIMEOUT;
-  __syncthreads();
-  return *slot != 0;
+// once instead of each waiting out its own limit.  Thread 0 alone reads the two words, once,
+// in its set-up block, and leaves the answer in `slot` (an int in shared memory); after the
+// kernel's first __syncthreads every thread reads the same answer there, whatever another
+// kernel writes to the status word in the meantime.
+__device__ __forceinline__ void note_skip(volatile int* slot, const int* status,
+                                          const int* abort_flag) {
+  *slot = (abort_flag && *(volatile const int*)abort_flag) ||
+          *(volatile const int*)status == SA_ERR_TIMEOUT;
 }
+// After that __syncthreads: leave (the allocating warp hands its tensor memory back first).
+#define SA_LEAVE_IF_SKIPPED(slot, alloc_warp, tmem, cols)                                     \
+  if (*(slot)) {                                                                              \
+    if (warp == (alloc_warp)) {                                                               \
+      tc_fence_after();                                                                       \
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem),       \
+                   "r"((uint32_t)(cols)) : "memory");                                         \
+    }                                                                                         \
+    return;                                                                                   \
+  }
 
 // Orders shared-memory writes made through the generic proxy (cp.async) that this thread
 // has observed before its later tensor-core reads of the same memory.
