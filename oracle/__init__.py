@@ -279,6 +279,36 @@ def backward_rows(q, k, v, perm, inv, gate_logits, dy, w, flags, q_rows, kv_rows
     return dq, dk, dv
 
 
+def rope(x, positions, base=10000.0, inverse=False):
+    """Rotary position embedding (Su et al.) of the last dimension of x, as the paper applies it
+    to Q and K BEFORE the shuffle, i.e. with each token's ORIGINAL position (Sec. 4.2 and the
+    attention paragraph of App. B).
+
+    x: [..., n, d] with d even; positions: [n] (the original token indices).  Dimension c of
+    the first half is paired with dimension c + d/2 (the half-split layout of the Qwen3 /
+    Llama family the paper retrofits; the adjacent-pair layout of the original formulation
+    differs only by a fixed permutation of the head dimensions).  The pair (x1, x2) of token
+    t is rotated by the angle positions[t] * base**(-2c/d):
+        out1 = x1 cos - x2 sin,   out2 = x2 cos + x1 sin.
+    inverse=True rotates by the opposite angle (the transpose: what maps a gradient with respect
+    to the rotated tensor back to the unrotated one).  Plain float64 numpy."""
+    x = np.asarray(x, dtype=np.float64)
+    d = x.shape[-1]
+    if d % 2:
+        raise ValueError("the head dimension must be even")
+    half = d // 2
+    pos = np.asarray(positions, dtype=np.float64)
+    if pos.shape != (x.shape[-2],):
+        raise ValueError("one position per token")
+    inv_freq = np.asarray(base, dtype=np.float64) ** (-2.0 * np.arange(half, dtype=np.float64) / d)
+    ang = pos[:, None] * inv_freq[None, :]
+    c, s = np.cos(ang), np.sin(ang)
+    if inverse:
+        s = -s
+    x1, x2 = x[..., :half], x[..., half:]
+    return np.concatenate([x1 * c - x2 * s, x2 * c + x1 * s], axis=-1)
+
+
 def gate_projection(y_sa, w_sa, y_swa=None, w_swa=None):
     """Projection gates of Eq. 5-6 (App. B, dual-path and single-path attention gate).
 
