@@ -481,6 +481,27 @@ def extras(args, c, wl, sa, torch, dev, host, perm, inv, ws, y, pk):
         del dyb, sv, bws3, bo
         torch.cuda.empty_cache()
 
+    # rotary position embedding with original positions (Sec. 4.2): rotation inside the gather
+    # of the SA forward against a rotation pass over Q and K followed by the plain forward
+    cs, sn = sa.sa_rope_table(c.n, c.d, 1e6)
+    qr, kr = torch.empty_like(q), torch.empty_like(k)
+    fused_ms = event_ms(lambda: sa.sa_forward_rope(q, k, v, perm, inv, cs, sn, c.w, c.flags, y=y),
+                        it, 3, torch)
+
+    def unfused():
+        sa.sa_rope_apply(q, k, cs, sn, out=qr)
+        sa.sa_rope_apply(k, q, cs, sn, out=kr, kv=True)
+        sa.sa_forward(qr, kr, v, perm, inv, c.w, c.flags, y=y)
+    unfused_ms = event_ms(unfused, it, 3, torch)
+    pass_ms = event_ms(lambda: (sa.sa_rope_apply(q, k, cs, sn, out=qr),
+                                sa.sa_rope_apply(k, q, cs, sn, out=kr, kv=True)), it, 3, torch)
+    res["rope"] = {"sa_fwd_rope_in_gather_ms": fused_ms, "rope_pass_plus_sa_fwd_ms": unfused_ms,
+                   "rope_pass_ms": pass_ms, "sa_fwd_ms": sa_ms,
+                   "pass_bytes": 2.0 * 2 * (q.numel() + k.numel()),
+                   "pass_gbs": 2.0 * 2 * (q.numel() + k.numel()) / (pass_ms * 1e-3) / 1e9}
+    del qr, kr, cs, sn
+    torch.cuda.empty_cache()
+
     # single-layer SA forward on the HBM-bound shape: tokens/s and the achieved bytes per second
     # over the algorithmic bytes (Q, K, V in, Y out, each once)
     c2 = wl.C2

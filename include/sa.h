@@ -76,7 +76,8 @@ typedef enum {
   SA_OP_GATED_FORWARD = 3,
   SA_OP_BACKWARD = 4,
   SA_OP_COVERAGE = 5,
-  SA_OP_GATED_FORWARD_SCRATCH = 6 /* optional scratch of sa_swa_gated_forward, see there */
+  SA_OP_GATED_FORWARD_SCRATCH = 6, /* optional scratch of sa_swa_gated_forward, see there */
+  SA_OP_FORWARD_ROPE = 7           /* sa_forward_rope / sa_swa_gated_forward_rope           */
 } sa_op;
 
 typedef struct {
@@ -189,6 +190,41 @@ sa_status sa_swa_gated_forward_host(const sa_problem* p, const void* q, const vo
  * their number, or -1 for bad head counts or too small an array. */
 int32_t sa_host_forward_plan(int32_t Hq, int32_t Hkv, int32_t n_groups, int32_t q_parts,
                              int32_t* pieces, int32_t max_pieces);
+
+/* Rotary position embedding with ORIGINAL token positions.  The paper applies RoPE to Q and K
+ * before the shuffle, with the positions the tokens have in the sequence, not the slots they
+ * are shuffled to (Sec. 4.2; attention paragraph of App. B).  Dimension c of the first half of
+ * a head is paired with dimension c + d/2 (the half-split layout of the Qwen3 / Llama family);
+ * token t turns the pair (x1, x2) by the angle t * base^(-2c/d):
+ *     out1 = x1 cos - x2 sin,   out2 = x2 cos + x1 sin      (fp32, rounded once to the dtype).
+ *
+ * sa_rope_table: rope_cos, rope_sin: out, device, fp32 [n, d/2]: cosine and sine of those
+ *   angles (angles in float64).  d even.
+ * sa_rope_apply: the rotation as a pass of its own.  x, out: device, [B,H,n,d] with the strides
+ *   of q (kv == 0: H = Hq) or of k (kv != 0: H = Hkv); out may be x.  inverse != 0 turns by the
+ *   opposite angle (the transpose: maps a gradient with respect to the rotated tensor back).
+ * sa_forward_rope / sa_swa_gated_forward_rope: sa_forward / sa_swa_gated_forward on rotated Q
+ *   and K without that pass: bf16 with d = 64 or 128 rotates the rows inside the kernels' row
+ *   gather, where the token a row belongs to is at hand (no rotated copy of Q or K exists);
+ *   every other case rotates Q and K into ws first (sa_workspace_bytes(.., SA_OP_FORWARD_ROPE)
+ *   bytes; 0 when the fused path applies).  Same results as sa_rope_apply followed by the plain
+ *   call.  For the backward pass rotate q and k with sa_rope_apply, call sa_backward on them, and
+ *   turn dq and dk back with inverse = 1.
+ * Errors: as the plain calls, plus SA_ERR_INVALID_ARG for null tables or odd d. */
+sa_status sa_rope_table(int32_t n, int32_t d, double base, float* rope_cos, float* rope_sin,
+                        sa_stream_t stream);
+sa_status sa_rope_apply(const sa_problem* p, int32_t kv, const void* x, const float* rope_cos,
+                        const float* rope_sin, int32_t inverse, void* out, sa_stream_t stream);
+sa_status sa_forward_rope(const sa_problem* p, const void* q, const void* k, const void* v,
+                          const int32_t* perm, const int32_t* inv, const float* rope_cos,
+                          const float* rope_sin, void* y, float* lse, void* ws, size_t ws_bytes,
+                          sa_stream_t stream);
+sa_status sa_swa_gated_forward_rope(const sa_problem* p, const void* q, const void* k,
+                                    const void* v, const int32_t* perm, const int32_t* inv,
+                                    const float* rope_cos, const float* rope_sin,
+                                    const float* gate_logits, void* y, void* y_sa, void* y_swa,
+                                    float* lse_sa, float* lse_swa, void* ws, size_t ws_bytes,
+                                    sa_stream_t stream);
 
 /* Backward of sa_forward (gate_logits == NULL: y_swa, lse_swa, dgate_logits ignored, y_sa
  * is the forward's y) or of sa_swa_gated_forward.  The paper only times this pass

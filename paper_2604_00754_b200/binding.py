@@ -31,7 +31,9 @@ EXPORTS = [
     "sa_gate_projection_forward", "sa_gate_projection_backward",
     "sa_gate_projection_backward_ws_bytes", "sa_debug_set", "sa_debug_wait_timeout",
     "sa_swa_gated_forward_host", "sa_host_forward_ws_bytes", "sa_host_forward_plan",
+    "sa_rope_table", "sa_rope_apply", "sa_forward_rope", "sa_swa_gated_forward_rope",
 ]
+OP_FORWARD_ROPE = 7
 DEBUG_SCORE_BLOCK, DEBUG_SWA_TILE_LOADS, DEBUG_TENSOR_CORES, DEBUG_GATE_WIDE_TILES = range(4)
 
 
@@ -110,6 +112,14 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     lib.sa_host_forward_plan.restype = i32
     lib.sa_swa_gated_forward_host.argtypes = [pp, vp, vp, vp, vp, vp, u64, u32, i32, i32, vp, sz, vp]
     lib.sa_swa_gated_forward_host.restype = ctypes.c_int
+    lib.sa_rope_table.argtypes = [i32, i32, ctypes.c_double, vp, vp, vp]
+    lib.sa_rope_table.restype = ctypes.c_int
+    lib.sa_rope_apply.argtypes = [pp, i32, vp, vp, vp, i32, vp, vp]
+    lib.sa_rope_apply.restype = ctypes.c_int
+    lib.sa_forward_rope.argtypes = [pp] + [vp] * 9 + [vp, sz, vp]
+    lib.sa_forward_rope.restype = ctypes.c_int
+    lib.sa_swa_gated_forward_rope.argtypes = [pp] + [vp] * 13 + [vp, sz, vp]
+    lib.sa_swa_gated_forward_rope.restype = ctypes.c_int
     lib.sa_debug_set.argtypes = [ctypes.c_int, ctypes.c_int]
     lib.sa_debug_set.restype = ctypes.c_int
     lib.sa_debug_wait_timeout.argtypes = [i64, vp]
@@ -267,6 +277,71 @@ def sa_swa_forward(q, k, v, w, flags=CAUSAL | SWA_ONE_SIDED, scale=0.0, y=None, 
     _check(lib.sa_swa_forward(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(y), _ptr(lse),
                               None, 0, _stream()), "sa_swa_forward")
     return (y, lse) if (want_lse or lse is not None) else y
+
+
+def sa_rope_table(n: int, d: int, base: float = 10000.0, device="cuda"):
+    """cos and sin of the rotary angles t * base^(-2c/d): fp32 [n, d/2] each."""
+    cs = torch.empty(n, d // 2, dtype=torch.float32, device=device)
+    sn = torch.empty_like(cs)
+    _check(load_library().sa_rope_table(n, d, float(base), _ptr(cs), _ptr(sn), _stream()),
+           "sa_rope_table")
+    return cs, sn
+
+
+def sa_rope_apply(x, k_like, rope_cos, rope_sin, w=1, inverse=False, out=None, kv=False):
+    """Rotates x ([B,H,n,d]) by its tokens' original positions; ``k_like`` is any tensor with the
+    KV layout (only needed to describe the problem when x is a query-side tensor)."""
+    q_like = k_like if kv else x
+    kv_like = x if kv else k_like
+    p = make_problem(q_like, kv_like, w, CAUSAL)
+    out = torch.empty_like(x) if out is None else out
+    _same_layout(x, out)
+    _check(load_library().sa_rope_apply(ctypes.byref(p), 1 if kv else 0, _ptr(x), _ptr(rope_cos),
+                                        _ptr(rope_sin), 1 if inverse else 0, _ptr(out), _stream()),
+           "sa_rope_apply")
+    return out
+
+
+def sa_forward_rope(q, k, v, perm, inv, rope_cos, rope_sin, w, flags=CAUSAL, scale=0.0, y=None,
+                    want_lse=False):
+    """SA forward on Q and K rotated by their original positions (rotation inside the gather
+    where the tensor-core kernels apply, a rotated copy in a workspace otherwise)."""
+    lib = load_library()
+    _same_layout(k, v)
+    p = make_problem(q, k, w, flags, scale)
+    y = torch.empty_like(q) if y is None else y
+    _same_layout(q, y)
+    lse = torch.empty(q.shape[:3], dtype=torch.float32, device=q.device) if want_lse else None
+    ws = _workspace(sa_workspace_bytes(p, OP_FORWARD_ROPE), q.device, None)
+    _check(lib.sa_forward_rope(ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(perm), _ptr(inv),
+                               _ptr(rope_cos), _ptr(rope_sin), _ptr(y), _ptr(lse), _ptr(ws),
+                               ws.numel(), _stream()), "sa_forward_rope")
+    return (y, lse) if want_lse else y
+
+
+def sa_swa_gated_forward_rope(q, k, v, perm, inv, rope_cos, rope_sin, gate_logits, w,
+                              flags=CAUSAL | SWA_ONE_SIDED, scale=0.0, save_for_bwd=False):
+    """Gated SA + SWA forward on rotated Q and K.  Returns y, or the five saved tensors."""
+    lib = load_library()
+    _same_layout(k, v)
+    out = {}
+    if save_for_bwd:
+        flags |= SAVE_FOR_BWD
+        for name in ("y_sa", "y_swa"):
+            out[name] = torch.empty_like(q)
+        for name in ("lse_sa", "lse_swa"):
+            out[name] = torch.empty(q.shape[:3], dtype=torch.float32, device=q.device)
+    y = torch.empty_like(q)
+    p = make_problem(q, k, w, flags, scale)
+    ws = _workspace(sa_workspace_bytes(p, OP_FORWARD_ROPE), q.device, None)
+    _check(lib.sa_swa_gated_forward_rope(
+        ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(perm), _ptr(inv), _ptr(rope_cos),
+        _ptr(rope_sin), _ptr(gate_logits), _ptr(y), _ptr(out.get("y_sa")), _ptr(out.get("y_swa")),
+        _ptr(out.get("lse_sa")), _ptr(out.get("lse_swa")), _ptr(ws), ws.numel(), _stream()),
+        "sa_swa_gated_forward_rope")
+    if save_for_bwd:
+        return y, out["y_sa"], out["y_swa"], out["lse_sa"], out["lse_swa"]
+    return y
 
 
 def sa_swa_gated_forward(q, k, v, perm, inv, gate_logits, w, flags=CAUSAL | SWA_ONE_SIDED,

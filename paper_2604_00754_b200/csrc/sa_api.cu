@@ -67,6 +67,14 @@ size_t branch_bytes(const sa_problem* p) {
   return (size_t)elems * (p->dtype == SA_BF16 ? 2 : 4);
 }
 
+// Bytes a tensor with the given strides spans (the rotated copies of the unfused RoPE path).
+size_t span_bytes(const sa_problem* p, bool kv) {
+  const int64_t* s = kv ? p->kv_stride : p->q_stride;
+  const int H = kv ? p->Hkv : p->Hq;
+  const int64_t elems = (p->B - 1) * s[0] + (H - 1) * s[1] + (int64_t)(p->n - 1) * s[2] + p->d;
+  return ((size_t)elems * (p->dtype == SA_BF16 ? 2 : 4) + 255) / 256 * 256;
+}
+
 float scale_of(const sa_problem* p) {
   return p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / std::sqrt((float)p->d);
 }
@@ -136,6 +144,12 @@ size_t sa_workspace_bytes(const sa_problem* p, int op) {
     case SA_OP_BACKWARD:
       if (check_problem(p) != SA_OK) return (size_t)-1;
       return bwd_ws_bytes(p->B, p->Hq, p->n, nullptr);
+    case SA_OP_FORWARD_ROPE: {
+      if (check_problem(p) != SA_OK || p->d % 2 != 0) return (size_t)-1;
+      FwdArgs a = fwd_args(p, p, p, p, false);      // pointers unused by the support test
+      if (tc_forward_supported(a, p->dtype)) return 0;
+      return span_bytes(p, false) + span_bytes(p, true);
+    }
     default:
       return (size_t)-1;
   }
@@ -228,6 +242,98 @@ sa_status sa_swa_gated_forward(const sa_problem* p, const void* q, const void* k
   FwdArgs a = fwd_args(p, q, k, v, false);
   a.perm = perm; a.inv = inv; a.y = y; a.y_branch = y_sa; a.lse = lse_sa;
   a.y_other = local_out; a.gate_logits = gate_logits;
+  return from_cuda(run_forward(a, p->dtype, st));
+}
+
+sa_status sa_rope_apply(const sa_problem* p, int32_t kv, const void* x, const float* rope_cos,
+                        const float* rope_sin, int32_t inverse, void* out, sa_stream_t stream) {
+  sa_status s = check_problem(p);
+  if (s != SA_OK) return s;
+  if (p->d % 2 != 0 || !good_ptr(x) || !good_ptr(out) || !rope_cos || !rope_sin)
+    return SA_ERR_INVALID_ARG;
+  return from_cuda(launch_rope_apply(x, out, p->B, kv ? p->Hkv : p->Hq, p->n, p->d,
+                                     kv ? p->kv_stride : p->q_stride, p->dtype, rope_cos,
+                                     rope_sin, inverse != 0, (cudaStream_t)stream));
+}
+
+namespace {
+// Where the fused rotation does not apply: rotated copies of q and k in the workspace.
+sa_status rope_prepass(const sa_problem* p, const void*& q, const void*& k, const float* rope_cos,
+                       const float* rope_sin, void* ws, size_t ws_bytes, cudaStream_t st) {
+  const size_t qb = span_bytes(p, false), kb = span_bytes(p, true);
+  if (!ws || !aligned16(ws)) return SA_ERR_INVALID_ARG;
+  if (ws_bytes < qb + kb) return SA_ERR_WORKSPACE;
+  void* qr = ws;
+  void* kr = (char*)ws + qb;
+  if (launch_rope_apply(q, qr, p->B, p->Hq, p->n, p->d, p->q_stride, p->dtype, rope_cos, rope_sin,
+                        false, st) != cudaSuccess ||
+      launch_rope_apply(k, kr, p->B, p->Hkv, p->n, p->d, p->kv_stride, p->dtype, rope_cos,
+                        rope_sin, false, st) != cudaSuccess)
+    return SA_ERR_CUDA;
+  q = qr;
+  k = kr;
+  return SA_OK;
+}
+}  // namespace
+
+sa_status sa_forward_rope(const sa_problem* p, const void* q, const void* k, const void* v,
+                          const int32_t* perm, const int32_t* inv, const float* rope_cos,
+                          const float* rope_sin, void* y, float* lse, void* ws, size_t ws_bytes,
+                          sa_stream_t stream) {
+  sa_status s = check_problem(p);
+  if (s != SA_OK) return s;
+  if (p->d % 2 != 0 || !rope_cos || !rope_sin || !aligned16(rope_cos) || !aligned16(rope_sin))
+    return SA_ERR_INVALID_ARG;
+  if (!good_ptr(q) || !good_ptr(k) || !good_ptr(v) || !good_ptr(perm) || !good_ptr(inv) ||
+      !good_ptr(y) || (lse && !aligned16(lse)))
+    return SA_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  if ((s = maybe_validate(p, perm, inv, st)) != SA_OK) return s;
+  FwdArgs a = fwd_args(p, q, k, v, false);
+  a.perm = perm; a.inv = inv; a.y = y; a.lse = lse;
+  if (tc_forward_supported(a, p->dtype)) {
+    a.rope_cos = rope_cos; a.rope_sin = rope_sin;
+  } else {
+    if ((s = rope_prepass(p, a.q, a.k, rope_cos, rope_sin, ws, ws_bytes, st)) != SA_OK) return s;
+  }
+  return from_cuda(run_forward(a, p->dtype, st));
+}
+
+sa_status sa_swa_gated_forward_rope(const sa_problem* p, const void* q, const void* k,
+                                    const void* v, const int32_t* perm, const int32_t* inv,
+                                    const float* rope_cos, const float* rope_sin,
+                                    const float* gate_logits, void* y, void* y_sa, void* y_swa,
+                                    float* lse_sa, float* lse_swa, void* ws, size_t ws_bytes,
+                                    sa_stream_t stream) {
+  sa_status s = check_problem(p);
+  if (s != SA_OK) return s;
+  if (p->d % 2 != 0 || !rope_cos || !rope_sin || !aligned16(rope_cos) || !aligned16(rope_sin))
+    return SA_ERR_INVALID_ARG;
+  if (!good_ptr(q) || !good_ptr(k) || !good_ptr(v) || !good_ptr(perm) || !good_ptr(inv) ||
+      !good_ptr(y) || !gate_logits)
+    return SA_ERR_INVALID_ARG;
+  if ((y_sa && !aligned16(y_sa)) || (y_swa && !aligned16(y_swa)) ||
+      (lse_sa && !aligned16(lse_sa)) || (lse_swa && !aligned16(lse_swa)))
+    return SA_ERR_INVALID_ARG;
+  if ((p->flags & SA_SAVE_FOR_BWD) && (!y_sa || !y_swa || !lse_sa || !lse_swa))
+    return SA_ERR_INVALID_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  if ((s = maybe_validate(p, perm, inv, st)) != SA_OK) return s;
+  FwdArgs probe = fwd_args(p, q, k, v, false);
+  const bool fused = tc_forward_supported(probe, p->dtype);
+  if (!fused && (s = rope_prepass(p, q, k, rope_cos, rope_sin, ws, ws_bytes, st)) != SA_OK)
+    return s;
+  // local branch first (its rows land in y_swa, or in y itself), then the SA branch, whose
+  // epilogue reads them back and applies both gates: the two-launch form of the gated forward
+  void* local_out = y_swa ? y_swa : y;
+  FwdArgs b = fwd_args(p, q, k, v, true);
+  b.y = nullptr; b.y_branch = local_out; b.lse = lse_swa;
+  if (fused) { b.rope_cos = rope_cos; b.rope_sin = rope_sin; }
+  if (run_forward(b, p->dtype, st) != cudaSuccess) return SA_ERR_CUDA;
+  FwdArgs a = fwd_args(p, q, k, v, false);
+  a.perm = perm; a.inv = inv; a.y = y; a.y_branch = y_sa; a.lse = lse_sa;
+  a.y_other = local_out; a.gate_logits = gate_logits;
+  if (fused) { a.rope_cos = rope_cos; a.rope_sin = rope_sin; }
   return from_cuda(run_forward(a, p->dtype, st));
 }
 

@@ -119,6 +119,7 @@ struct FwdArgs {
   void* y_branch;             // nullable: this branch's own (ungated) output
   float* lse;                 // nullable
   const void* y_other;        // nullable: the other branch's finished output (gated combine)
+  const float *rope_cos, *rope_sin;  // nullable [n, d/2]: rotate Q and K rows inside the gather
   const float* gate_logits;   // nullable [2,Hq]
   int B, Hq, Hkv, n, d, w;
   uint32_t flags;
@@ -155,6 +156,10 @@ size_t make_perm_ws_bytes(int B, int n);
 cudaError_t launch_fwd_simt(const FwdArgs& a, int dtype, cudaStream_t st);
 cudaError_t launch_validate_perm(const int32_t* perm, const int32_t* inv, int B, int n,
                                  cudaStream_t st);
+
+cudaError_t launch_rope_apply(const void* x, void* out, int B, int H, int n, int d,
+                              const int64_t s[3], int dtype, const float* cs, const float* sn,
+                              bool inverse, cudaStream_t st);
 
 cudaError_t launch_combine(void* y, const void* y_sa, const void* y_swa, const float* logits,
                            int B, int Hq, int n, int d, const int64_t s[3], int dtype,

@@ -43,6 +43,7 @@ enum TileClass { kSkip = 0, kFull = 1, kCausalOnly = 2, kEdge = 3 };
 struct TcParams {
   const void *q, *k, *v;
   const int32_t* perm;        // null for the SWA branch
+  const float *rope_cos, *rope_sin;   // null, or [n, D/2] each: rotate Q and K rows on the way in
   void* y;
   void* y_branch;
   const void* y_other;
@@ -191,7 +192,9 @@ struct Cfg {
 // two blocks and the scores run two blocks ahead of the softmax; with 128 a block is the
 // whole K/V tile and the next scores of a tile follow its P V.
 // TMA: the instantiation for launches whose tiles come by TMA (p.use_tma).
-template <int D, int KB, bool TMA>
+// ROPE: the gather producers rotate the rows of Q and K by their tokens' angles (rotary
+// position embedding with ORIGINAL positions, Sec. 4.2 / App. B) after the copies have landed.
+template <int D, int KB, bool TMA, bool ROPE = false>
 __global__ void __launch_bounds__(kThreads, 1)
 fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtensorMap tm_q,
               const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v) {
@@ -239,7 +242,11 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
   // (12 x 168).  The four warps of a warpgroup must ask for the same count, so the issuing
   // warp and the producer warps go down together.  With 224 registers the 128 scores and the
   // 32 packed probabilities of a softmax thread stay in registers (at 208 they spilled).
-  asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
+  // With ROPE the producers need room for the rotation: 4 x 72 + 8 x 216 = 2016 again.  (The
+  // sum may never exceed what the launch holds: a warpgroup asking for more waits for ever.)
+  static_assert(4 * 72 + 8 * 216 == 12 * 168 && 4 * 56 + 8 * 224 == 12 * 168, "register split");
+  if (ROPE) asm volatile("setmaxnreg.dec.sync.aligned.u32 72;");
+  else asm volatile("setmaxnreg.dec.sync.aligned.u32 56;");
   if (warp >= 1 && TMA) {
     // ------------------------------------------- tile loads by TMA (one thread of warp 1)
     // Rows are consecutive tokens here, so a tile is D / 64 boxes of 128 tokens x 64 columns
@@ -386,6 +393,53 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
       return any != 0;
     };
 
+    // ROPE: rows of a landed tile that this warp copied are turned in place.  A lane owns the
+    // 16-byte piece `chunk` of its rows; the piece half a row further on holds the partner
+    // dimensions (c <-> c + D/2).  Every lane reads both pieces, the warp meets, every lane
+    // writes its own piece back: out = own * cos -/+ partner * sin (first / second half), in
+    // fp32, rounded once to bf16 -- the arithmetic of the stand-alone rotation pass.
+    auto rotate = [&](const int32_t* toks, uint32_t tile) {
+      constexpr int kHalfC = kCpr / 2;
+      const int pc = chunk < kHalfC ? chunk + kHalfC : chunk - kHalfC;
+      const int fc = chunk < kHalfC ? chunk : chunk - kHalfC;
+      const float sgn = chunk < kHalfC ? -1.f : 1.f;
+      for (int grp = warp - 1; grp < kGroups; grp += 3) {
+        const int r = grp * kRpi + sub;
+        const uint32_t rb = tile + r * 128;
+        const uint32_t a_own = rb + (uint32_t)(chunk >> 3) * C::kChunkBytes +
+                               (uint32_t)(((chunk & 7) ^ (r & 7)) << 4);
+        const uint32_t a_oth = rb + (uint32_t)(pc >> 3) * C::kChunkBytes +
+                               (uint32_t)(((pc & 7) ^ (r & 7)) << 4);
+        uint32_t own[4], oth[4];
+        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(own[0]), "=r"(own[1]), "=r"(own[2]), "=r"(own[3]) : "r"(a_own) : "memory");
+        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(oth[0]), "=r"(oth[1]), "=r"(oth[2]), "=r"(oth[3]) : "r"(a_oth) : "memory");
+        const size_t at = (size_t)toks[r] * (D / 2) + 8 * fc;
+        __syncwarp();
+        uint32_t res[4];
+#pragma unroll
+        for (int hx = 0; hx < 2; ++hx) {           // four dimensions at a time: few live registers
+          const float4 c4 = *reinterpret_cast<const float4*>(p.rope_cos + at + 4 * hx);
+          const float4 s4 = *reinterpret_cast<const float4*>(p.rope_sin + at + 4 * hx);
+          const float co[4] = {c4.x, c4.y, c4.z, c4.w}, si[4] = {s4.x, s4.y, s4.z, s4.w};
+#pragma unroll
+          for (int x = 0; x < 2; ++x) {
+            const int w = 2 * hx + x;
+            const float2 o = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&own[w]));
+            const float2 t = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&oth[w]));
+            const __nv_bfloat162 h2 = __floats2bfloat162_rn(
+                fmaf(o.x, co[2 * x], sgn * (t.x * si[2 * x])),
+                fmaf(o.y, co[2 * x + 1], sgn * (t.y * si[2 * x + 1])));
+            res[w] = *reinterpret_cast<const uint32_t*>(&h2);
+          }
+        }
+        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};"
+                     ::"r"(a_own), "r"(res[0]), "r"(res[1]), "r"(res[2]), "r"(res[3]) : "memory");
+      }
+    };
+    auto commit_group = [&]() { asm volatile("cp.async.commit_group;" ::: "memory"); };
+
     bool live = true;
     for (int w_item = blockIdx.x; w_item < p.total_items && live; w_item += gridDim.x, ++it) {
       const int item = w_item % p.items_per_kv, bh = w_item / p.items_per_kv;
@@ -414,8 +468,10 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
         if (ptid < 32) ktok[ptid + 96] = tk1;
         if (group_sync_stop()) { live = false; break; }
         if (ptid == 0) mbar_arrive(bar(C::kBarTokFull + gt % C::kTok));
-        gather(kb, p.ks[2], ktok, sbase + C::kOffRing + (use % C::kSlots) * C::kTileBytes);
-        signal(bar(C::kBarSlotFull + use % C::kSlots));
+        const uint32_t k_dst = sbase + C::kOffRing + (use % C::kSlots) * C::kTileBytes;
+        const uint32_t k_bar = bar(C::kBarSlotFull + use % C::kSlots);
+        gather(kb, p.ks[2], ktok, k_dst);
+        if (ROPE) commit_group(); else signal(k_bar);
         ++use;
         if (j + 1 < g.T) {
           tk0 = key_tok(j + 1, ptid);
@@ -432,7 +488,7 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
           for (int t = 0; t < 2; ++t)
             gather(qg + b * p.qs[0] + g.hq[t] * p.qs[1], p.qs[2], qtok + t * kTile,
                    sbase + C::kOffQ + t * C::kTileBytes);
-          signal(bar(C::kBarQFull));
+          if (ROPE) commit_group(); else signal(bar(C::kBarQFull));
         }
         // ---- V_j
         if (use >= (uint32_t)C::kSlots)
@@ -441,6 +497,21 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
         gather(vb, p.ks[2], ktok, sbase + C::kOffRing + (use % C::kSlots) * C::kTileBytes);
         signal(bar(C::kBarSlotFull + use % C::kSlots));
         ++use;
+        if (ROPE) {
+          // K_j (and Q at the start of an item) have landed once at most the V_j copies are
+          // still under way; turn the rows, publish them to the tensor core's proxy, arrive
+          commit_group();
+          asm volatile("cp.async.wait_group 1;" ::: "memory");
+          __syncwarp();
+          rotate(ktok, k_dst);
+          if (j == 0) {
+            rotate(qtok, sbase + C::kOffQ);
+            rotate(qtok + kTile, sbase + C::kOffQ + C::kTileBytes);
+          }
+          fence_proxy_async();
+          mbar_arrive(k_bar);
+          if (j == 0) mbar_arrive(bar(C::kBarQFull));
+        }
       }
     }
     asm volatile("cp.async.wait_all;" ::: "memory");   // nothing in flight when the CTA leaves
@@ -561,7 +632,8 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
     __syncwarp();
   }
   } else {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
+    if (ROPE) asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
+    else asm volatile("setmaxnreg.inc.sync.aligned.u32 224;");
     // ------------------------------------------------- softmax and epilogue
     const int t = (warp - 4) / 4;
     const int row = threadIdx.x - 128 - t * 128;       // 0..127 == TMEM lane
@@ -838,6 +910,7 @@ cudaError_t launch_fwd_tc(const FwdArgs& a, cudaStream_t st) {
   TcParams p{};
   p.q = a.q; p.k = a.k; p.v = a.v;
   p.perm = a.swa ? nullptr : a.perm;
+  p.rope_cos = a.rope_cos; p.rope_sin = a.rope_sin;
   p.y = a.y; p.y_branch = a.y_branch; p.y_other = a.y_other; p.lse = a.lse;
   p.gate_logits = a.gate_logits;
   p.status = status_ptr();
@@ -868,7 +941,7 @@ cudaError_t launch_fwd_tc(const FwdArgs& a, cudaStream_t st) {
   // whole-tile TMA loads for the one-sided SWA branch (any strides the maps can express;
   // otherwise the gather serves this branch too)
   CUtensorMap tm_q{}, tm_k{}, tm_v{};
-  if (a.swa && mg.one_sided && !swa_tma_disabled()) {
+  if (a.swa && mg.one_sided && !swa_tma_disabled() && !a.rope_cos) {   // TMA tiles cannot be turned
     if (aligned16(a.q) && aligned16(a.k) && aligned16(a.v) &&
         make_map_bhnd(&tm_q, a.q, a.B, a.Hq, a.n, a.d, a.qs) &&
         make_map_bhnd(&tm_k, a.k, a.B, a.Hkv, a.n, a.d, a.ks) &&
@@ -882,7 +955,12 @@ cudaError_t launch_fwd_tc(const FwdArgs& a, cudaStream_t st) {
     return cudaSuccess;
   };
   const bool tma = p.use_tma != 0;
-  if (a.d == 128)
+  if (a.rope_cos)
+    e = a.d == 128 ? (wide ? go(fwd_tc_kernel<128, 128, false, true>, Cfg<128>::kBytes)
+                           : go(fwd_tc_kernel<128, 64, false, true>, Cfg<128>::kBytes))
+                   : (wide ? go(fwd_tc_kernel<64, 128, false, true>, Cfg<64>::kBytes)
+                           : go(fwd_tc_kernel<64, 64, false, true>, Cfg<64>::kBytes));
+  else if (a.d == 128)
     e = wide ? (tma ? go(fwd_tc_kernel<128, 128, true>, Cfg<128>::kBytes)
                     : go(fwd_tc_kernel<128, 128, false>, Cfg<128>::kBytes))
              : (tma ? go(fwd_tc_kernel<128, 64, true>, Cfg<128>::kBytes)

@@ -91,3 +91,31 @@ def test_rope_rejects_bad_shapes():
         oracle.rope(np.zeros((3, 5)), np.arange(3))
     with pytest.raises(ValueError):
         oracle.rope(np.zeros((3, 4)), np.arange(2))
+
+
+def test_gradient_through_the_rotation_by_finite_differences():
+    """d/dq and d/dk of sum(dy * SA(rope(q), rope(k), v)) is the inverse rotation (the
+    transpose) of the gradient with respect to the rotated tensors."""
+    rng = np.random.default_rng(4)
+    B, H, n, d, w = 1, 2, 10, 4, 5
+    q, k, v = (rng.standard_normal((B, H, n, d)) for _ in range(3))
+    dy = rng.standard_normal((B, H, n, d))
+    perm, inv = oracle.make_perm(6, 0, B, n)
+    pos = np.arange(n)
+    f = lambda q_, k_: float((dy * oracle.sa_forward(oracle.rope(q_, pos), oracle.rope(k_, pos), v,
+                                                     perm, inv, w, CAUSAL)[0]).sum())
+    gq, gk, _, _ = oracle.backward(oracle.rope(q, pos), oracle.rope(k, pos), v, perm, inv, None, dy,
+                                   w, CAUSAL)
+    dq, dk = oracle.rope(gq, pos, inverse=True), oracle.rope(gk, pos, inverse=True)
+    eps = 1e-6
+    for arr, grad, which in ((q, dq, 0), (k, dk, 1)):
+        flat = arr.reshape(-1)
+        for e in rng.choice(flat.size, size=20, replace=False):
+            old = flat[e]
+            flat[e] = old + eps
+            lp = f(q, k)
+            flat[e] = old - eps
+            lm = f(q, k)
+            flat[e] = old
+            fd = (lp - lm) / (2 * eps)
+            assert abs(fd - grad.reshape(-1)[e]) <= 1e-7 * max(1.0, abs(fd)), (which, e)
