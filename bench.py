@@ -187,6 +187,10 @@ def main():
     ap.add_argument("--score-block", type=int, default=0, choices=[0, 64, 128],
                     help="force the score-block width of the tensor-core kernels (test hook of "
                          "the library; 0 = the library's own choice)")
+    ap.add_argument("--gated-form", default="streaming", choices=["epilogue", "streaming"],
+                    help="how the gates are applied: in the local branch's epilogue (two launches, "
+                         "what the library does without scratch) or by a third, streaming kernel given "
+                         "scratch (faster at this size: the default here)")
     ap.add_argument("--no-extras", action="store_true",
                     help="skip the side measurements (SWA, backward, e2e, CPU oracle)")
     args = ap.parse_args()
@@ -248,7 +252,8 @@ def main():
 
     def step():
         sa.sa_make_perm(cr.seed, layer[0], c.B, c.n, perm=perm, inv=inv, ws=ws)
-        sa.sa_swa_gated_forward(q, k, v, perm, inv, lg, c.w, c.flags, out=out, ws=gws)
+        sa.sa_swa_gated_forward(q, k, v, perm, inv, lg, c.w, c.flags, out=out,
+                                ws=gws if args.gated_form == "streaming" else None)
         layer[0] += 1
 
     def barrier():
@@ -307,7 +312,9 @@ def main():
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic", "config": workload_config(c), "clocks": clocks,
         "gpu_launches": int(launches),
-        "roofline": {"kernel": "fused SA forward (gather, QK^T, softmax, PV, scatter); a streaming kernel applies the gates to both branches afterwards",
+        "roofline": {"kernel": "fused SA forward (gather, QK^T, softmax, PV, scatter); the gates are applied "
+                               + ("by a streaming kernel afterwards" if args.gated_form == "streaming"
+                                  else "in the epilogue of the local branch's launch"),
                      "bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                      "frac": achieved / peak,
                      "peak_kind": "%s bf16 %s" % (pk["source"], "sustained" if sustained else "burst"),

@@ -150,12 +150,13 @@ sa_status sa_swa_forward(const sa_problem* p, const void* q, const void* k, cons
  * y = sigmoid(gate_logits[0,hq]) * y_sa + sigmoid(gate_logits[1,hq]) * y_swa.
  * y: out.  y_sa, y_swa, lse_sa, lse_swa: out, nullable unless SA_SAVE_FOR_BWD; the
  * branch outputs are stored in the run dtype before they are combined.
- * ws is optional (sa_workspace_bytes(.., SA_OP_GATED_FORWARD) is 0).  When ws holds at least
- * sa_workspace_bytes(.., SA_OP_GATED_FORWARD_SCRATCH) bytes (one branch output in q's
- * layout), or y_swa is given and a branch output is 64 MB or more, the branches run ungated
- * and a streaming kernel combines them, which is faster for large outputs; otherwise the SA
- * branch's epilogue reads the local branch's rows and combines.  Same result either way up
- * to the rounding of the branch outputs to the run dtype. */
+ * ws is optional (sa_workspace_bytes(.., SA_OP_GATED_FORWARD) is 0).  Without it the call is
+ * two launches: the SA branch writes its ungated rows (to y_sa, or to y itself), then the local
+ * branch, whose rows are consecutive tokens, reads them back in its epilogue, applies both
+ * gates and writes y.  When ws holds at least sa_workspace_bytes(.., SA_OP_GATED_FORWARD_SCRATCH)
+ * bytes (one branch output in q's layout) both branches run ungated and a third, streaming
+ * kernel combines them.  Same result either way up to the rounding of the local branch's
+ * output to the run dtype before it is combined (done when it is stored). */
 sa_status sa_swa_gated_forward(const sa_problem* p, const void* q, const void* k,
                                const void* v, const int32_t* perm, const int32_t* inv,
                                const float* gate_logits, void* y, void* y_sa, void* y_swa,

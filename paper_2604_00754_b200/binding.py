@@ -349,9 +349,10 @@ def sa_swa_gated_forward(q, k, v, perm, inv, gate_logits, w, flags=CAUSAL | SWA_
     """Gated SA + SWA forward.  Returns y, or (y, y_sa, y_swa, lse_sa, lse_swa) when saving.
 
     ``out`` may hold preallocated tensors under the keys y, y_sa, y_swa, lse_sa, lse_swa.
-    ``ws``: optional scratch (uint8) for the local branch's rows when y_swa is not kept; one is
-    allocated when it is missing, unless ``fused_epilogue`` asks for the path that needs none
-    (the SA launch's epilogue then does the combination)."""
+    ``ws``: optional scratch (uint8, OP_GATED_FORWARD_SCRATCH bytes): with it the branches run
+    ungated and a streaming kernel combines them (three launches); without it the local
+    branch's epilogue does the combination (two launches).  ``fused_epilogue=True`` drops a
+    given ``ws``."""
     lib = load_library()
     _same_layout(k, v)
     out = dict(out or {})
@@ -366,11 +367,6 @@ def sa_swa_gated_forward(q, k, v, perm, inv, gate_logits, w, flags=CAUSAL | SWA_
     p = make_problem(q, k, w, flags, scale)
     if fused_epilogue:
         ws = None
-    elif ws is None and out.get("y_swa") is None:
-        # worth a scratch tensor and a third launch only when the outputs are large
-        nbytes = sa_workspace_bytes(p, OP_GATED_FORWARD_SCRATCH)
-        if nbytes >= (64 << 20):
-            ws = _workspace(nbytes, q.device, None)
     _check(lib.sa_swa_gated_forward(
         ctypes.byref(p), _ptr(q), _ptr(k), _ptr(v), _ptr(perm), _ptr(inv), _ptr(gate_logits),
         _ptr(y), _ptr(out.get("y_sa")), _ptr(out.get("y_swa")), _ptr(out.get("lse_sa")),

@@ -210,15 +210,10 @@ sa_status sa_swa_gated_forward(const sa_problem* p, const void* q, const void* k
     return SA_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   if ((s = maybe_validate(p, perm, inv, st)) != SA_OK) return s;
-  // With room for the local branch's rows (the caller's y_swa, or scratch) both branches run
-  // ungated and a streaming kernel combines them: cheaper than reading the other branch's
-  // row inside the attention epilogue, where the loads sit on the softmax warps' path.
-  // Scratch says the caller wants this path; with only y_swa to go by it is taken for large
-  // outputs (measured: from about 64 MB per branch the third launch costs less than the
-  // epilogue loads; below, e.g. the 50 MB of the pre-training shape, it does not).
-  const bool scratch = ws && ws_bytes >= branch_bytes(p);
-  void* swa_rows = y_swa ? y_swa : (scratch ? ws : nullptr);
-  if (swa_rows && (scratch || branch_bytes(p) >= ((size_t)64 << 20))) {
+  // With scratch for one branch output the caller asks for the three-launch form: both branches
+  // ungated, then a streaming kernel that applies the gates.
+  if (ws && ws_bytes >= branch_bytes(p)) {
+    void* swa_rows = y_swa ? y_swa : ws;
     void* sa_rows = y_sa ? y_sa : y;
     FwdArgs a = fwd_args(p, q, k, v, false);
     a.perm = perm; a.inv = inv; a.y = sa_rows; a.lse = lse_sa;
@@ -231,18 +226,21 @@ sa_status sa_swa_gated_forward(const sa_problem* p, const void* q, const void* k
     return from_cuda(launch_combine(y, sa_rows, swa_rows, gate_logits, p->B, p->Hq, p->n, p->d,
                                     p->q_stride, p->dtype, st));
   }
-  // Without it, local branch first: its rows land in y_swa (or in y itself when the caller does not keep
-  // them).  The SA branch then owns each output row exactly once: it reads the local
-  // branch's row, applies both gates and writes y.
-  void* local_out = y_swa ? y_swa : y;
-  FwdArgs b = fwd_args(p, q, k, v, true);
-  b.y = nullptr; b.y_branch = local_out; b.lse = lse_swa;
-  cudaError_t e = run_forward(b, p->dtype, st);
-  if (e != cudaSuccess) return SA_ERR_CUDA;
+  // Otherwise two launches.  The SA branch first: its ungated rows land in y_sa, or in y itself
+  // when the caller does not keep them.  The local branch then owns each output row exactly
+  // once: its rows are consecutive tokens, so the matching SA rows are read back as one
+  // contiguous run per query tile, both gates are applied and y is written.  (Reading the
+  // scattered rows of the local branch from the SA branch's epilogue, the other possible order,
+  // costs more than a third launch.)
+  void* sa_rows = y_sa ? y_sa : y;
   FwdArgs a = fwd_args(p, q, k, v, false);
-  a.perm = perm; a.inv = inv; a.y = y; a.y_branch = y_sa; a.lse = lse_sa;
-  a.y_other = local_out; a.gate_logits = gate_logits;
-  return from_cuda(run_forward(a, p->dtype, st));
+  a.perm = perm; a.inv = inv; a.y = sa_rows; a.lse = lse_sa;
+  cudaError_t e = run_forward(a, p->dtype, st);
+  if (e != cudaSuccess) return SA_ERR_CUDA;
+  FwdArgs b = fwd_args(p, q, k, v, true);
+  b.y = y; b.y_branch = y_swa; b.lse = lse_swa;
+  b.y_other = sa_rows; b.gate_logits = gate_logits;
+  return from_cuda(run_forward(b, p->dtype, st));
 }
 
 sa_status sa_rope_apply(const sa_problem* p, int32_t kv, const void* x, const float* rope_cos,
@@ -323,18 +321,17 @@ sa_status sa_swa_gated_forward_rope(const sa_problem* p, const void* q, const vo
   const bool fused = tc_forward_supported(probe, p->dtype);
   if (!fused && (s = rope_prepass(p, q, k, rope_cos, rope_sin, ws, ws_bytes, st)) != SA_OK)
     return s;
-  // local branch first (its rows land in y_swa, or in y itself), then the SA branch, whose
-  // epilogue reads them back and applies both gates: the two-launch form of the gated forward
-  void* local_out = y_swa ? y_swa : y;
-  FwdArgs b = fwd_args(p, q, k, v, true);
-  b.y = nullptr; b.y_branch = local_out; b.lse = lse_swa;
-  if (fused) { b.rope_cos = rope_cos; b.rope_sin = rope_sin; }
-  if (run_forward(b, p->dtype, st) != cudaSuccess) return SA_ERR_CUDA;
+  // SA branch first, the local branch combines (see sa_swa_gated_forward)
+  void* sa_rows = y_sa ? y_sa : y;
   FwdArgs a = fwd_args(p, q, k, v, false);
-  a.perm = perm; a.inv = inv; a.y = y; a.y_branch = y_sa; a.lse = lse_sa;
-  a.y_other = local_out; a.gate_logits = gate_logits;
+  a.perm = perm; a.inv = inv; a.y = sa_rows; a.lse = lse_sa;
   if (fused) { a.rope_cos = rope_cos; a.rope_sin = rope_sin; }
-  return from_cuda(run_forward(a, p->dtype, st));
+  if (run_forward(a, p->dtype, st) != cudaSuccess) return SA_ERR_CUDA;
+  FwdArgs b = fwd_args(p, q, k, v, true);
+  b.y = y; b.y_branch = y_swa; b.lse = lse_swa;
+  b.y_other = sa_rows; b.gate_logits = gate_logits;
+  if (fused) { b.rope_cos = rope_cos; b.rope_sin = rope_sin; }
+  return from_cuda(run_forward(b, p->dtype, st));
 }
 
 sa_status sa_backward(const sa_problem* p, const void* q, const void* k, const void* v,

@@ -194,7 +194,10 @@ struct Cfg {
 // TMA: the instantiation for launches whose tiles come by TMA (p.use_tma).
 // ROPE: the gather producers rotate the rows of Q and K by their tokens' angles (rotary
 // position embedding with ORIGINAL positions, Sec. 4.2 / App. B) after the copies have landed.
-template <int D, int KB, bool TMA, bool ROPE = false>
+// COMBINE: the epilogue reads the other branch's finished rows and applies the gates of Eq. 5
+// (the instantiation of the launch that closes a gated forward); without it the kernel
+// carries no gate code at all.
+template <int D, int KB, bool TMA, bool ROPE = false, bool COMBINE = false>
 __global__ void __launch_bounds__(kThreads, 1)
 fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtensorMap tm_q,
               const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v) {
@@ -677,7 +680,7 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
       const bool row_valid = cur.row_valid;
       const int q_tok = cur.q_tok;
       const int qcmp = (p.causal && !p.one_sided) ? q_tok : 0x7fffffff;
-      if (p.gate_logits && p.y_other && row_valid) {
+      if (COMBINE && row_valid) {
         // the epilogue will read the other branch's row: start bringing it into L2 now
         const __nv_bfloat16* orow = (const __nv_bfloat16*)p.y_other + b * p.qs[0] +
                                     cur.hq * p.qs[1] + (int64_t)q_tok * p.qs[2];
@@ -810,7 +813,7 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
       const float inv_l = 1.f / l;
       float g_this = 1.f, g_other = 0.f;
       const int hq = cur.hq;
-      if (p.gate_logits) {
+      if (COMBINE) {
         const float s_sa = 1.f / (1.f + __expf(-p.gate_logits[hq]));
         const float s_swa = 1.f / (1.f + __expf(-p.gate_logits[p.Hq + hq]));
         g_this = p.swa ? s_swa : s_sa;
@@ -821,6 +824,17 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
       for (int c = 0; c < D / 32; ++c) {
         uint32_t raw[32];
         tmem_ld32(o_addr + 32 * c, raw);       // warp-collective: every lane takes part
+        // Gated combine: this piece of the other branch's row (in L2 since the start of the
+        // item) is requested before anything of the piece is stored, four loads in flight
+        // together.  y may be the buffer the other rows sit in: a piece is read before the
+        // same columns are written.
+        uint4 oth[4];
+        if (COMBINE && row_valid) {
+#pragma unroll
+          for (int x8 = 0; x8 < 4; ++x8)
+            oth[x8] = *reinterpret_cast<const uint4*>((const __nv_bfloat16*)p.y_other + off +
+                                                      32 * c + 8 * x8);
+        }
         tmem_wait_ld();
         if (row_valid) {
 #pragma unroll
@@ -840,17 +854,12 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
               }
               *reinterpret_cast<uint4*>((__nv_bfloat16*)p.y_branch + e) = st;
             }
-            if (p.gate_logits) {
+            if (COMBINE) {
+              const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&oth[x8]);
 #pragma unroll
-              for (int x = 0; x < 8; ++x) o[x] *= g_this;
-              if (p.y_other) {
-                const uint4 ot = *reinterpret_cast<const uint4*>((const __nv_bfloat16*)p.y_other + e);
-                const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&ot);
-#pragma unroll
-                for (int x = 0; x < 4; ++x) {
-                  o[2 * x] = fmaf(g_other, __low2float(h2[x]), o[2 * x]);
-                  o[2 * x + 1] = fmaf(g_other, __high2float(h2[x]), o[2 * x + 1]);
-                }
+              for (int x = 0; x < 4; ++x) {
+                o[2 * x] = fmaf(g_other, __low2float(h2[x]), o[2 * x] * g_this);
+                o[2 * x + 1] = fmaf(g_other, __high2float(h2[x]), o[2 * x + 1] * g_this);
               }
             }
             if (p.y) {
@@ -955,21 +964,24 @@ cudaError_t launch_fwd_tc(const FwdArgs& a, cudaStream_t st) {
     return cudaSuccess;
   };
   const bool tma = p.use_tma != 0;
-  if (a.rope_cos)
-    e = a.d == 128 ? (wide ? go(fwd_tc_kernel<128, 128, false, true>, Cfg<128>::kBytes)
-                           : go(fwd_tc_kernel<128, 64, false, true>, Cfg<128>::kBytes))
-                   : (wide ? go(fwd_tc_kernel<64, 128, false, true>, Cfg<64>::kBytes)
-                           : go(fwd_tc_kernel<64, 64, false, true>, Cfg<64>::kBytes));
-  else if (a.d == 128)
-    e = wide ? (tma ? go(fwd_tc_kernel<128, 128, true>, Cfg<128>::kBytes)
-                    : go(fwd_tc_kernel<128, 128, false>, Cfg<128>::kBytes))
-             : (tma ? go(fwd_tc_kernel<128, 64, true>, Cfg<128>::kBytes)
-                    : go(fwd_tc_kernel<128, 64, false>, Cfg<128>::kBytes));
-  else
-    e = wide ? (tma ? go(fwd_tc_kernel<64, 128, true>, Cfg<64>::kBytes)
-                    : go(fwd_tc_kernel<64, 128, false>, Cfg<64>::kBytes))
-             : (tma ? go(fwd_tc_kernel<64, 64, true>, Cfg<64>::kBytes)
-                    : go(fwd_tc_kernel<64, 64, false>, Cfg<64>::kBytes));
+  const bool combine = a.gate_logits && a.y_other;
+  if (a.gate_logits && !a.y_other) return cudaErrorInvalidValue;   // gates only with the other rows
+  // instantiation by (head dimension, score-block width, tile loads, rotation, combine)
+  auto pick = [&](auto d_c, auto kb_c) {
+    constexpr int DD = decltype(d_c)::value, KK = decltype(kb_c)::value;
+    if (a.rope_cos)
+      return combine ? go(fwd_tc_kernel<DD, KK, false, true, true>, Cfg<DD>::kBytes)
+                     : go(fwd_tc_kernel<DD, KK, false, true, false>, Cfg<DD>::kBytes);
+    if (tma)
+      return combine ? go(fwd_tc_kernel<DD, KK, true, false, true>, Cfg<DD>::kBytes)
+                     : go(fwd_tc_kernel<DD, KK, true, false, false>, Cfg<DD>::kBytes);
+    return combine ? go(fwd_tc_kernel<DD, KK, false, false, true>, Cfg<DD>::kBytes)
+                   : go(fwd_tc_kernel<DD, KK, false, false, false>, Cfg<DD>::kBytes);
+  };
+  using I64 = std::integral_constant<int, 64>;
+  using I128 = std::integral_constant<int, 128>;
+  if (a.d == 128) e = wide ? pick(I128{}, I128{}) : pick(I128{}, I64{});
+  else e = wide ? pick(I64{}, I128{}) : pick(I64{}, I64{});
   if (e != cudaSuccess) return e;
   bump_launches();
   return cudaGetLastError();
