@@ -562,7 +562,10 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
         mma_ts_x4(tmem + C::kColO + t * D, tmem + t * 128 + b * kHalf, vd, idesc_pv, acc0);
         if (KB == 128)
           mma_ts_x4(tmem + C::kColO + t * D, tmem + t * 128 + 32, vd + 512, idesc_pv, 1u);
-        tc_commit(bar(C::kBarPvDone + t));
+        // A commit holds the tensor pipe up for some 180 cycles, so none is spent where another
+        // one already tells the same: with 128-key blocks the next scores of this tile follow
+        // this product in the pipe, and their "S full" says that it is over as well.
+        if (NB == 2) tc_commit(bar(C::kBarPvDone + t));
       };
       for (int w_item = blockIdx.x; w_item < p.total_items && ok; w_item += gridDim.x, ++it) {
         const int item = w_item % p.items_per_kv, bh = w_item / p.items_per_kv;
@@ -760,10 +763,13 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
           m = m_new;
         } else if (__any_sync(0xffffffffu, grow)) {
           // O is still being accumulated by the previous P V: wait for it before touching O
-          ok = mbar_wait(bar(C::kBarPvDone + t), (pv_cnt - 1) & 1u, gave_up, p.status);
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) break;
-          tc_fence_after();
+          // (128-key blocks: these scores were issued behind that product, so it is over)
+          if (NB == 2) {
+            ok = mbar_wait(bar(C::kBarPvDone + t), (pv_cnt - 1) & 1u, gave_up, p.status);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+          }
           const float f = grow ? exp2f((m - m_new) * p.scale2) : 1.f;
           if (grow) { l *= f; m = m_new; }
 #pragma unroll
