@@ -4,7 +4,8 @@
 One step = one pass of the forward hot path over one batch of the Qwen3-8B-shaped
 workload (bf16, B=1, 32 query / 8 KV heads, d=128, n=32768, w=1024): a fresh permutation
 (sa_make_perm) followed by the gated SA+SWA forward (sa_swa_gated_forward), which runs the
-fused SA kernel, the plain SWA kernel and the streaming gate-and-combine kernel.  `value` is tokens/s of that step.
+fused SA kernel and then the plain SWA kernel, whose launch also applies the gates and
+combines the two branches.  `value` is tokens/s of that step.
 Beside it the JSON line reports the SA-only and SWA-only forward (tokens/s, TFLOP/s with
 4*B*Hq*n*w*d nominal flops, SA overhead over SWA), the permutation alone, the backward on
 the pre-training shape, a roofline entry for the SA forward kernel timed live with CUDA
@@ -187,10 +188,10 @@ def main():
     ap.add_argument("--score-block", type=int, default=0, choices=[0, 64, 128],
                     help="force the score-block width of the tensor-core kernels (test hook of "
                          "the library; 0 = the library's own choice)")
-    ap.add_argument("--gated-form", default="streaming", choices=["epilogue", "streaming"],
-                    help="how the gates are applied: in the local branch's epilogue (two launches, "
-                         "what the library does without scratch) or by a third, streaming kernel given "
-                         "scratch (faster at this size: the default here)")
+    ap.add_argument("--gated-form", default="warps", choices=["warps", "epilogue"],
+                    help="where the local branch's launch applies the gates: in its two idle warps "
+                         "(scratch for the SA rows given: the default) or in the row threads' "
+                         "epilogue (no scratch)")
     ap.add_argument("--no-extras", action="store_true",
                     help="skip the side measurements (SWA, backward, e2e, CPU oracle)")
     args = ap.parse_args()
@@ -231,7 +232,7 @@ def main():
     prob = sa.SaProblem(B=c.B, n=c.n)
     ws = torch.empty(sa.sa_workspace_bytes(prob, sa.OP_MAKE_PERM), dtype=torch.uint8, device="cuda")
     out = {"y": y}
-    # scratch for the local branch's rows: the gates are then applied by a streaming kernel
+    # scratch for the SA branch's rows: the local branch's launch then combines with its idle warps
     gws = torch.empty(sa.sa_workspace_bytes(sa.make_problem(q, k, c.w, c.flags),
                                             sa.OP_GATED_FORWARD_SCRATCH),
                       dtype=torch.uint8, device="cuda")
@@ -253,7 +254,7 @@ def main():
     def step():
         sa.sa_make_perm(cr.seed, layer[0], c.B, c.n, perm=perm, inv=inv, ws=ws)
         sa.sa_swa_gated_forward(q, k, v, perm, inv, lg, c.w, c.flags, out=out,
-                                ws=gws if args.gated_form == "streaming" else None)
+                                ws=gws if args.gated_form == "warps" else None)
         layer[0] += 1
 
     def barrier():
@@ -313,7 +314,8 @@ def main():
         "data": "synthetic", "config": workload_config(c), "clocks": clocks,
         "gpu_launches": int(launches),
         "roofline": {"kernel": "fused SA forward (gather, QK^T, softmax, PV, scatter); the gates are applied "
-                               + ("by a streaming kernel afterwards" if args.gated_form == "streaming"
+                               + ("by two idle warps of the local branch's launch"
+                                  if args.gated_form == "warps"
                                   else "in the epilogue of the local branch's launch"),
                      "bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                      "frac": achieved / peak,

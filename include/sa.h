@@ -150,13 +150,14 @@ sa_status sa_swa_forward(const sa_problem* p, const void* q, const void* k, cons
  * y = sigmoid(gate_logits[0,hq]) * y_sa + sigmoid(gate_logits[1,hq]) * y_swa.
  * y: out.  y_sa, y_swa, lse_sa, lse_swa: out, nullable unless SA_SAVE_FOR_BWD; the
  * branch outputs are stored in the run dtype before they are combined.
- * ws is optional (sa_workspace_bytes(.., SA_OP_GATED_FORWARD) is 0).  Without it the call is
- * two launches: the SA branch writes its ungated rows (to y_sa, or to y itself), then the local
- * branch, whose rows are consecutive tokens, reads them back in its epilogue, applies both
- * gates and writes y.  When ws holds at least sa_workspace_bytes(.., SA_OP_GATED_FORWARD_SCRATCH)
- * bytes (one branch output in q's layout) both branches run ungated and a third, streaming
- * kernel combines them.  Same result either way up to the rounding of the local branch's
- * output to the run dtype before it is combined (done when it is stored). */
+ * Two launches: the SA branch writes its ungated rows (to y_sa, else to ws, else to y itself),
+ * then the local branch, whose rows are consecutive tokens, reads them back, applies both
+ * gates and writes y.  ws is optional (sa_workspace_bytes(.., SA_OP_GATED_FORWARD) is 0): with
+ * at least sa_workspace_bytes(.., SA_OP_GATED_FORWARD_SCRATCH) bytes (one branch output in
+ * q's layout) a caller that keeps neither branch output still gets the faster form of the
+ * combination, in which the local branch stores its rows (rounded to the run dtype) and two
+ * otherwise idle warps of the same launch combine them; without any such buffer the row
+ * threads combine in their epilogue, from unrounded local rows. */
 sa_status sa_swa_gated_forward(const sa_problem* p, const void* q, const void* k,
                                const void* v, const int32_t* perm, const int32_t* inv,
                                const float* gate_logits, void* y, void* y_sa, void* y_swa,
@@ -170,8 +171,8 @@ sa_status sa_swa_gated_forward(const sa_problem* p, const void* q, const void* k
  * travel through the GPU in n_groups contiguous ranges (a range of one KV head in q_parts
  * ranges of its query heads when they divide evenly), on three internal streams: copy in,
  * compute, copy out.  The permutation is drawn from (seed, layer) as in sa_make_perm and
- * shared by all ranges; the gates are applied by the streaming combine of
- * sa_swa_gated_forward, so the result has the bits of that call given scratch.
+ * shared by all ranges; every range is one sa_swa_gated_forward call given scratch, so the
+ * result has the bits of that call.
  *   ws: DEVICE workspace of sa_host_forward_ws_bytes(p) bytes, 256-byte aligned, owned by the
  *       caller (device copies of q, k, v, y, one branch output, the permutation and its
  *       scratch).  No device memory is allocated; the first call on a device creates the

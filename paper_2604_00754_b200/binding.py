@@ -349,10 +349,10 @@ def sa_swa_gated_forward(q, k, v, perm, inv, gate_logits, w, flags=CAUSAL | SWA_
     """Gated SA + SWA forward.  Returns y, or (y, y_sa, y_swa, lse_sa, lse_swa) when saving.
 
     ``out`` may hold preallocated tensors under the keys y, y_sa, y_swa, lse_sa, lse_swa.
-    ``ws``: optional scratch (uint8, OP_GATED_FORWARD_SCRATCH bytes): with it the branches run
-    ungated and a streaming kernel combines them (three launches); without it the local
-    branch's epilogue does the combination (two launches).  ``fused_epilogue=True`` drops a
-    given ``ws``."""
+    ``ws``: optional scratch (uint8, OP_GATED_FORWARD_SCRATCH bytes) for the SA branch's rows
+    when neither branch output is kept: the local branch's launch then combines with its idle
+    warps instead of in the row threads' epilogue.  ``fused_epilogue=True`` drops a given
+    ``ws``.  Two launches either way."""
     lib = load_library()
     _same_layout(k, v)
     out = dict(out or {})

@@ -210,29 +210,16 @@ sa_status sa_swa_gated_forward(const sa_problem* p, const void* q, const void* k
     return SA_ERR_INVALID_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   if ((s = maybe_validate(p, perm, inv, st)) != SA_OK) return s;
-  // With scratch for one branch output the caller asks for the three-launch form: both branches
-  // ungated, then a streaming kernel that applies the gates.
-  if (ws && ws_bytes >= branch_bytes(p)) {
-    void* swa_rows = y_swa ? y_swa : ws;
-    void* sa_rows = y_sa ? y_sa : y;
-    FwdArgs a = fwd_args(p, q, k, v, false);
-    a.perm = perm; a.inv = inv; a.y = sa_rows; a.lse = lse_sa;
-    cudaError_t e = run_forward(a, p->dtype, st);
-    if (e != cudaSuccess) return SA_ERR_CUDA;
-    FwdArgs b = fwd_args(p, q, k, v, true);
-    b.y = swa_rows; b.lse = lse_swa;
-    e = run_forward(b, p->dtype, st);
-    if (e != cudaSuccess) return SA_ERR_CUDA;
-    return from_cuda(launch_combine(y, sa_rows, swa_rows, gate_logits, p->B, p->Hq, p->n, p->d,
-                                    p->q_stride, p->dtype, st));
-  }
-  // Otherwise two launches.  The SA branch first: its ungated rows land in y_sa, or in y itself
-  // when the caller does not keep them.  The local branch then owns each output row exactly
-  // once: its rows are consecutive tokens, so the matching SA rows are read back as one
-  // contiguous run per query tile, both gates are applied and y is written.  (Reading the
-  // scattered rows of the local branch from the SA branch's epilogue, the other possible order,
-  // costs more than a third launch.)
-  void* sa_rows = y_sa ? y_sa : y;
+  // Two launches.  The SA branch first: its ungated rows land in y_sa, else in the scratch,
+  // else in y itself.  The local branch then owns each output row exactly once and its rows
+  // are consecutive tokens, so the matching SA rows are read back as contiguous runs, both
+  // gates are applied and y is written: by the two warps that have nothing to load when the
+  // local branch's tiles come by TMA (this needs a home for the local rows other than the
+  // buffer the SA rows sit in: y_swa, or y when the SA rows are elsewhere), otherwise in the
+  // row threads' epilogue.  (Reading the scattered rows of the local branch from the SA
+  // branch's epilogue, the other possible order, costs more than a third launch would.)
+  const bool scratch = ws && ws_bytes >= branch_bytes(p);
+  void* sa_rows = y_sa ? y_sa : (scratch ? ws : y);
   FwdArgs a = fwd_args(p, q, k, v, false);
   a.perm = perm; a.inv = inv; a.y = sa_rows; a.lse = lse_sa;
   cudaError_t e = run_forward(a, p->dtype, st);

@@ -161,10 +161,6 @@ cudaError_t launch_rope_apply(const void* x, void* out, int B, int H, int n, int
                               const int64_t s[3], int dtype, const float* cs, const float* sn,
                               bool inverse, cudaStream_t st);
 
-cudaError_t launch_combine(void* y, const void* y_sa, const void* y_swa, const float* logits,
-                           int B, int Hq, int n, int d, const int64_t s[3], int dtype,
-                           cudaStream_t st);
-
 bool gate_forward_wide(int64_t rows, int dm, const void* y_sa, const void* y_swa, int64_t ld_y,
                        const void* w_sa, const void* w_swa, void* out, int64_t ld_out,
                        int* status, int sms, cudaStream_t st, cudaError_t* err);

@@ -179,7 +179,8 @@ struct Cfg {
                        kBarSlotEmpty = kBarSlotFull + kSlots, kBarTokFull = kBarSlotEmpty + kSlots,
                        kBarSFull = kBarTokFull + kTok, kBarPReady = kBarSFull + 4,
                        kBarPvDone = kBarPReady + 4, kBarODone = kBarPvDone + 2,
-                       kNumBars = kBarODone + 2;
+                       kBarRowsDone = kBarODone + 2, kBarRowsTaken = kBarRowsDone + 2,
+                       kNumBars = kBarRowsTaken + 2;
   static constexpr int kOffMisc = kOffBar + kNumBars * 8;   // TMEM base address, gave_up flag
   static constexpr int kBytes = kOffMisc + 16;
   static constexpr uint32_t kColO = 256;                     // O_t at 256 + t*D; S_t at t*128
@@ -222,7 +223,8 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
     *gave_up = 0;
     note_skip(reinterpret_cast<volatile int*>(smem + C::kOffMisc + 8), p.status, p.abort_flag);
     for (int i = 0; i < C::kNumBars; ++i)
-      mbar_init(bar(i), (i >= C::kBarPReady && i < C::kBarPvDone) ? kTile
+      mbar_init(bar(i), i >= C::kBarRowsTaken ? 64      // the two combining warps
+                        : ((i >= C::kBarPReady && i < C::kBarPvDone) || i >= C::kBarRowsDone) ? kTile
                         : (i == C::kBarQFull || (i >= C::kBarSlotFull && i < C::kBarSlotEmpty))
                             ? (p.use_tma ? 1 : kProducers) : 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -318,6 +320,87 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
             if (mbar_try(bar(C::kBarQFull), q_armed & 1u)) break;
             __nanosleep(100);
           }
+      }
+    } else if (COMBINE && warp >= 2) {
+      // ------------------------------- gated combine by the two idle warps (Eq. 5)
+      // With tiles coming by TMA, warps 2 and 3 have nothing to load.  The row threads store
+      // this branch's finished rows ungated (to y_branch, else to y) and arrive on "rows
+      // done"; these 64 threads then read them back together with the other branch's rows
+      // (both from L2), apply the two gates and write y, 16 bytes per thread and step, off
+      // the row threads' path.  Each 16-byte piece is read and written by one thread, so y
+      // may be the buffer this branch's rows were stored in.  "Rows taken" tells the row
+      // threads that their previous arrival has been seen, so that the two barriers can
+      // never be a whole phase apart (a one-bit parity could not tell).
+      constexpr int kCpr = D / 8, kRowsPerPass = 64 / kCpr;
+      const int ctid = threadIdx.x - 64, chunk = ctid % kCpr, rsub = ctid / kCpr;
+      const __nv_bfloat16* mine = (const __nv_bfloat16*)(p.y_branch ? p.y_branch : p.y);
+      const __nv_bfloat16* other = (const __nv_bfloat16*)p.y_other;
+      __nv_bfloat16* yout = (__nv_bfloat16*)p.y;
+      uint32_t done0 = 0, done1 = 0;
+      bool live = true;
+      for (int w_item = blockIdx.x; w_item < p.total_items && live; w_item += gridDim.x) {
+        const int item = w_item % p.items_per_kv, bh = w_item / p.items_per_kv;
+        const int b = bh / p.Hkv;
+        const Geo g = make_geo(p, item, bh % p.Hkv);
+        // the other branch's rows of this item will be wanted a whole item from now: start
+        // bringing them into L2 (one 128-byte line per thread and step)
+#pragma unroll 1
+        for (int t = 0; t < 2; ++t) {
+          if (!g.valid[t]) continue;
+          const __nv_bfloat16* ob = other + b * p.qs[0] + g.hq[t] * p.qs[1];
+          for (int x = ctid; x < kTile * (D / 64); x += 64) {
+            const int slot = g.q0[t] + x / (D / 64);
+            if (slot < p.n)
+              asm volatile("prefetch.global.L2 [%0];" ::"l"(ob + (int64_t)slot * p.qs[2] + 64 * (x % (D / 64))));
+          }
+        }
+#pragma unroll 1
+        for (int t = 0; t < 2 && live; ++t) {
+          if (!g.valid[t]) continue;
+          live = mbar_wait(bar(C::kBarRowsDone + t), (t ? done1 : done0) & 1u, gave_up, p.status);
+          if (!live) break;
+          mbar_arrive(bar(C::kBarRowsTaken + t));
+          done0 += 1 - t;
+          done1 += t;
+          const int hq = g.hq[t];
+          const float g_sa = 1.f / (1.f + __expf(-p.gate_logits[hq]));
+          const float g_swa = 1.f / (1.f + __expf(-p.gate_logits[p.Hq + hq]));
+          const float g_mine = p.swa ? g_swa : g_sa, g_oth = p.swa ? g_sa : g_swa;
+          const int64_t base = b * p.qs[0] + hq * p.qs[1] + chunk * 8;
+#pragma unroll 1
+          for (int r0 = rsub; r0 < kTile; r0 += 4 * kRowsPerPass) {
+            uint4 a[4], c4[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              const int slot = g.q0[t] + r0 + u * kRowsPerPass;   // this branch: token == slot
+              if (slot < p.n) {
+                const int64_t off = base + (int64_t)slot * p.qs[2];
+                a[u] = __ldcg(reinterpret_cast<const uint4*>(mine + off));
+                c4[u] = __ldcg(reinterpret_cast<const uint4*>(other + off));
+              }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              const int slot = g.q0[t] + r0 + u * kRowsPerPass;
+              if (slot < p.n) {
+                const __nv_bfloat162* hm = reinterpret_cast<const __nv_bfloat162*>(&a[u]);
+                const __nv_bfloat162* ho = reinterpret_cast<const __nv_bfloat162*>(&c4[u]);
+                uint4 o;
+                __nv_bfloat162* hr = reinterpret_cast<__nv_bfloat162*>(&o);
+                // sa term times its gate first, then the local term by fma
+                const float gs = p.swa ? g_oth : g_mine, gl = p.swa ? g_mine : g_oth;
+#pragma unroll
+                for (int x = 0; x < 4; ++x) {
+                  const __nv_bfloat162 sa2 = p.swa ? ho[x] : hm[x], lo2 = p.swa ? hm[x] : ho[x];
+                  hr[x] = __floats2bfloat162_rn(
+                      fmaf(gl, __low2float(lo2), gs * __low2float(sa2)),
+                      fmaf(gl, __high2float(lo2), gs * __high2float(sa2)));
+                }
+                *reinterpret_cast<uint4*>(yout + base + (int64_t)slot * p.qs[2]) = o;
+              }
+            }
+          }
+        }
       }
     }
   } else if (warp >= 1 && !TMA) {
@@ -646,7 +729,7 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
     const uint32_t lane_addr = (uint32_t)(row & ~31) << 16;
     const uint32_t s_addr = tmem + lane_addr + t * 128;
     const uint32_t o_addr = tmem + lane_addr + C::kColO + t * D;
-    uint32_t s_cnt0 = 0, s_cnt1 = 0, o_cnt = 0, pv_cnt = 0, gt = 0;
+    uint32_t s_cnt0 = 0, s_cnt1 = 0, o_cnt = 0, pv_cnt = 0, gt = 0, rows_cnt = 0;
     bool ok = true;
 
     // geometry and query token of an item; fetched one item ahead
@@ -683,7 +766,7 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
       const bool row_valid = cur.row_valid;
       const int q_tok = cur.q_tok;
       const int qcmp = (p.causal && !p.one_sided) ? q_tok : 0x7fffffff;
-      if (COMBINE && row_valid) {
+      if (COMBINE && !TMA && row_valid) {
         // the epilogue will read the other branch's row: start bringing it into L2 now
         const __nv_bfloat16* orow = (const __nv_bfloat16*)p.y_other + b * p.qs[0] +
                                     cur.hq * p.qs[1] + (int64_t)q_tok * p.qs[2];
@@ -819,7 +902,8 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
       const float inv_l = 1.f / l;
       float g_this = 1.f, g_other = 0.f;
       const int hq = cur.hq;
-      if (COMBINE) {
+      constexpr bool wc = COMBINE && TMA;   // with TMA tiles the gates are applied by warps 2 and 3
+      if (COMBINE && !wc) {
         const float s_sa = 1.f / (1.f + __expf(-p.gate_logits[hq]));
         const float s_swa = 1.f / (1.f + __expf(-p.gate_logits[p.Hq + hq]));
         g_this = p.swa ? s_swa : s_sa;
@@ -835,7 +919,7 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
         // together.  y may be the buffer the other rows sit in: a piece is read before the
         // same columns are written.
         uint4 oth[4];
-        if (COMBINE && row_valid) {
+        if (COMBINE && !wc && row_valid) {
 #pragma unroll
           for (int x8 = 0; x8 < 4; ++x8)
             oth[x8] = *reinterpret_cast<const uint4*>((const __nv_bfloat16*)p.y_other + off +
@@ -860,7 +944,7 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
               }
               *reinterpret_cast<uint4*>((__nv_bfloat16*)p.y_branch + e) = st;
             }
-            if (COMBINE) {
+            if (COMBINE && !wc) {
               const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&oth[x8]);
 #pragma unroll
               for (int x = 0; x < 4; ++x) {
@@ -868,7 +952,7 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
                 o[2 * x + 1] = fmaf(g_other, __high2float(h2[x]), o[2 * x + 1] * g_this);
               }
             }
-            if (p.y) {
+            if (p.y && !(wc && p.y_branch)) {   // (wc: y is written by the combining warps)
               uint4 st;
               __nv_bfloat162* h2 = reinterpret_cast<__nv_bfloat162*>(&st);
 #pragma unroll
@@ -880,6 +964,15 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
       }
       if (p.lse && row_valid)
         p.lse[((size_t)b * p.Hq + hq) * p.n + q_tok] = (m * p.scale2 + log2f(l)) * kLn2;
+      // rows of this tile are stored: the combining warps may take them (release at CTA scope),
+      // once they have seen the arrival for the item before
+      if (wc) {
+        if (rows_cnt) ok = mbar_wait(bar(C::kBarRowsTaken + t), (rows_cnt - 1) & 1u, gave_up, p.status);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        mbar_arrive(bar(C::kBarRowsDone + t));
+        ++rows_cnt;
+      }
       // the next item's first P V overwrites O: order these reads before the arrive that
       // lets it start
       tc_fence_before();
@@ -956,7 +1049,10 @@ cudaError_t launch_fwd_tc(const FwdArgs& a, cudaStream_t st) {
   // whole-tile TMA loads for the one-sided SWA branch (any strides the maps can express;
   // otherwise the gather serves this branch too)
   CUtensorMap tm_q{}, tm_k{}, tm_v{};
-  if (a.swa && mg.one_sided && !swa_tma_disabled() && !a.rope_cos) {   // TMA tiles cannot be turned
+  const bool rows_have_a_home =
+      !(a.gate_logits && a.y_other) || (a.y_branch ? a.y_branch != a.y_other : a.y != a.y_other);
+  if (a.swa && mg.one_sided && !swa_tma_disabled() && !a.rope_cos &&   // TMA tiles cannot be turned
+      rows_have_a_home) {
     if (aligned16(a.q) && aligned16(a.k) && aligned16(a.v) &&
         make_map_bhnd(&tm_q, a.q, a.B, a.Hq, a.n, a.d, a.qs) &&
         make_map_bhnd(&tm_k, a.k, a.B, a.Hkv, a.n, a.d, a.ks) &&
@@ -971,6 +1067,8 @@ cudaError_t launch_fwd_tc(const FwdArgs& a, cudaStream_t st) {
   };
   const bool tma = p.use_tma != 0;
   const bool combine = a.gate_logits && a.y_other;
+  // (checked below: the TMA variant combines with its idle warps, which needs this branch's rows
+  // to have a home that is not the buffer the other branch's rows sit in)
   if (a.gate_logits && !a.y_other) return cudaErrorInvalidValue;   // gates only with the other rows
   // instantiation by (head dimension, score-block width, tile loads, rotation, combine)
   auto pick = [&](auto d_c, auto kb_c) {

@@ -67,7 +67,7 @@ def test_pipelined_forward_equals_single_call(n_groups, q_parts):
     hf.forward(q, k, v, lg, hy, seed=5, layer=2)
     torch.cuda.synchronize()
     perm, inv = sa.sa_make_perm(5, 2, B, n)
-    # the pipeline hands the library scratch, so its gates are applied by the streaming
+    # the pipeline hands the library scratch, so its gates are applied by the idle-warp
     # kernel: the single call does the same (the fused epilogue rounds differently)
     scratch = torch.empty(hy.numel() * hy.element_size(), dtype=torch.uint8, device="cuda")
     ref = sa.sa_swa_gated_forward(q.cuda(), k.cuda(), v.cuda(), perm, inv, lg.cuda(), w, ws=scratch)
