@@ -79,10 +79,14 @@ __device__ __forceinline__ int actual_slot(const BwdTcParams& p, int v) {
   return v < 0 ? v + p.n : v;
 }
 
-template <int D, int KC, int MODE, int NBUF>
+// RW: warpgroups of row threads.  Two split a column tile's 32-column pieces between them: with
+// two score buffers (products of the next tile overlap the row work) or, for 128-wide tiles,
+// with one buffer, where they halve the time the tensor core waits for the row threads.
+template <int D, int KC, int MODE, int NBUF, int RW>
 struct BCfg {
   static_assert(NBUF == 1 || KC == 64, "two score buffers need 64-wide column tiles");
-  static constexpr int kRowWgs = NBUF;                          // warpgroups of row threads
+  static_assert(RW == 1 || RW == 2, "one or two warpgroups of row threads");
+  static constexpr int kRowWgs = RW;                            // warpgroups of row threads
   static constexpr int kThreads = 128 + 128 * kRowWgs;
   static constexpr int kTileBytes = kTile * D * 2;              // a row-operand tile
   static constexpr int kChunkBytes = kTile * 128;               // its 64-column blocks
@@ -111,11 +115,12 @@ struct BCfg {
 };
 
 // MODE 0: rows are queries (dQ).  MODE 1: rows are keys (dK, dV).
-template <int D, int KC, int MODE, int NBUF>
-__global__ void __launch_bounds__(BCfg<D, KC, MODE, NBUF>::kThreads, BCfg<D, KC, MODE, NBUF>::kCtasPerSm)
+template <int D, int KC, int MODE, int NBUF, int RW>
+__global__ void __launch_bounds__(BCfg<D, KC, MODE, NBUF, RW>::kThreads,
+                                  BCfg<D, KC, MODE, NBUF, RW>::kCtasPerSm)
 bwd_tc_kernel(const __grid_constant__ BwdTcParams p) {
   extern __shared__ __align__(1024) uint8_t smem[];
-  using C = BCfg<D, KC, MODE, NBUF>;
+  using C = BCfg<D, KC, MODE, NBUF, RW>;
   constexpr uint32_t kTmemCols = C::kTmemCols;
   constexpr bool kKeys = MODE == 1;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -217,23 +222,32 @@ bwd_tc_kernel(const __grid_constant__ BwdTcParams p) {
       }
       signal(bar(C::kBarRFull));
     }
+    // The tokens of a column tile come from global memory (perm); they are fetched one tile
+    // ahead of their use so that this latency is not paid inside every step.
+    auto col_tok = [&](int it, int x) {
+      const int j = kKeys ? it % T : it;
+      return tok_of(actual_slot(p, cstart + j * KC + x));
+    };
+    int nt0 = 0, nt1 = 0;
+    if (live && iters > 0) {
+      if (ptid < KC) nt0 = col_tok(0, ptid);
+      if (ptid + 96 < KC) nt1 = col_tok(0, ptid + 96);
+    }
     for (int it = 0; it < iters && live; ++it) {
       const int s = it % C::kStages;
-      const int j = kKeys ? it % T : it, gi = kKeys ? it / T : 0;
+      const int gi = kKeys ? it / T : 0;
       const int hq = kKeys ? hk * p.G + gi : hr;
+      const int t0 = nt0, t1 = nt1;
+      if (it + 1 < iters) {
+        if (ptid < KC) nt0 = col_tok(it + 1, ptid);
+        if (ptid + 96 < KC) nt1 = col_tok(it + 1, ptid + 96);
+      }
       if (it >= C::kStages)
         mbar_wait(bar(C::kBarCEmpty + s), (it / C::kStages - 1) & 1u, gave_up, p.status);
       int32_t* coltok = reinterpret_cast<int32_t*>(smem + C::kOffColTok) + s * kTile;
       const uint32_t colvec = sbase + C::kOffColVec + s * 2 * kTile * 4;
-      int t0 = 0, t1 = 0;
-      if (ptid < KC) {
-        t0 = tok_of(actual_slot(p, cstart + j * KC + ptid));
-        coltok[ptid] = t0;
-      }
-      if (ptid + 96 < KC) {
-        t1 = tok_of(actual_slot(p, cstart + j * KC + ptid + 96));
-        coltok[ptid + 96] = t1;
-      }
+      if (ptid < KC) coltok[ptid] = t0;
+      if (ptid + 96 < KC) coltok[ptid + 96] = t1;
       if (group_sync_stop()) { live = false; break; }
       if (ptid == 0) mbar_arrive(bar(C::kBarTokFull + s));
       const uint32_t c1 = sbase + C::kOffC + s * 2 * C::kColBytes, c2 = c1 + C::kColBytes;
@@ -515,30 +529,34 @@ bwd_tc_kernel(const __grid_constant__ BwdTcParams p) {
 
 // ---------------------------------------------------------------------------- host
 
-template <int D, int KC, int NBUF>
+template <int D, int KC, int NBUF, int RW>
 cudaError_t launch_branch(const BwdTcParams& p, cudaStream_t st) {
-  using C0 = BCfg<D, KC, 0, NBUF>;
-  using C1 = BCfg<D, KC, 1, NBUF>;
-  cudaError_t e = cudaFuncSetAttribute(bwd_tc_kernel<D, KC, 0, NBUF>,
+  using C0 = BCfg<D, KC, 0, NBUF, RW>;
+  using C1 = BCfg<D, KC, 1, NBUF, RW>;
+  cudaError_t e = cudaFuncSetAttribute(bwd_tc_kernel<D, KC, 0, NBUF, RW>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, C0::kBytes);
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(bwd_tc_kernel<D, KC, 1, NBUF>,
+  e = cudaFuncSetAttribute(bwd_tc_kernel<D, KC, 1, NBUF, RW>,
                            cudaFuncAttributeMaxDynamicSharedMemorySize, C1::kBytes);
   if (e != cudaSuccess) return e;
-  bwd_tc_kernel<D, KC, 0, NBUF><<<(unsigned)(p.B * p.Hq * p.n_tiles), C0::kThreads, C0::kBytes, st>>>(p);
-  bwd_tc_kernel<D, KC, 1, NBUF><<<(unsigned)(p.B * p.Hkv * p.n_tiles), C1::kThreads, C1::kBytes, st>>>(p);
+  bwd_tc_kernel<D, KC, 0, NBUF, RW><<<(unsigned)(p.B * p.Hq * p.n_tiles), C0::kThreads, C0::kBytes, st>>>(p);
+  bwd_tc_kernel<D, KC, 1, NBUF, RW><<<(unsigned)(p.B * p.Hkv * p.n_tiles), C1::kThreads, C1::kBytes, st>>>(p);
   bump_launches(2);
   return cudaGetLastError();
 }
 
+constexpr int kWideDefault = 1;   // shape for w > 128
+
 // Kernel shape: 0 = 64-wide column tiles, one score buffer (narrow windows: least band-edge
 // waste, two CTAs per SM at d = 64); 1 = 64-wide tiles, two score buffers and two row
 // warpgroups (products of the next tile overlap the row work of this one); 2 = 128-wide
-// tiles, one buffer.  sa_debug_set(SA_DEBUG_SCORE_BLOCK, 64 | 128) forces shape 0 or 2.
+// tiles, one buffer, two row warpgroups (a third fewer tensor-pipe cycles per column than
+// 64-wide tiles, and half the wait for the row threads).
+// sa_debug_set(SA_DEBUG_SCORE_BLOCK, 64 | 128) forces shape 0 or 2.
 int bwd_shape(int w) {
   const int forced = debug_option(SA_DEBUG_SCORE_BLOCK);
   if (forced) return forced == 64 ? 0 : 2;
-  return w <= 128 ? 0 : 1;
+  return w <= 128 ? 0 : kWideDefault;
 }
 
 bool bwd_tc_disabled() { return debug_option(SA_DEBUG_TENSOR_CORES) == 0; }
@@ -575,11 +593,11 @@ cudaError_t launch_bwd_tc(const BwdArgs& a, cudaStream_t st) {
     const int shape = bwd_shape(a.w);
     cudaError_t e;
     if (a.d == 128)
-      e = shape == 0 ? launch_branch<128, 64, 1>(p, st)
-          : shape == 1 ? launch_branch<128, 64, 2>(p, st) : launch_branch<128, 128, 1>(p, st);
+      e = shape == 0 ? launch_branch<128, 64, 1, 1>(p, st)
+          : shape == 1 ? launch_branch<128, 64, 2, 2>(p, st) : launch_branch<128, 128, 1, 2>(p, st);
     else
-      e = shape == 0 ? launch_branch<64, 64, 1>(p, st)
-          : shape == 1 ? launch_branch<64, 64, 2>(p, st) : launch_branch<64, 128, 1>(p, st);
+      e = shape == 0 ? launch_branch<64, 64, 1, 1>(p, st)
+          : shape == 1 ? launch_branch<64, 64, 2, 2>(p, st) : launch_branch<64, 128, 1, 2>(p, st);
     if (e != cudaSuccess) return e;
   }
   return cudaSuccess;
