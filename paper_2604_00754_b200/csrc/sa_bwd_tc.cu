@@ -32,6 +32,7 @@
 #include <type_traits>
 
 #include "sa_bwd_tc.cuh"
+#include "sa_gemm_common.cuh"
 #include "sa_tc_common.cuh"
 
 namespace sa {
@@ -115,10 +116,15 @@ struct BCfg {
 };
 
 // MODE 0: rows are queries (dQ).  MODE 1: rows are keys (dK, dV).
-template <int D, int KC, int MODE, int NBUF, int RW>
+// TMA: the instantiation for the one-sided SWA branch, whose rows are consecutive tokens: one
+// warp loads whole tiles with cp.async.bulk.tensor (no multicast) instead of three warps
+// gathering rows 16 bytes at a time, which is bound by the load/store unit.
+template <int D, int KC, int MODE, int NBUF, int RW, bool TMA>
 __global__ void __launch_bounds__(BCfg<D, KC, MODE, NBUF, RW>::kThreads,
                                   BCfg<D, KC, MODE, NBUF, RW>::kCtasPerSm)
-bwd_tc_kernel(const __grid_constant__ BwdTcParams p) {
+bwd_tc_kernel(const __grid_constant__ BwdTcParams p, const __grid_constant__ CUtensorMap tm_q,
+              const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+              const __grid_constant__ CUtensorMap tm_dy) {
   extern __shared__ __align__(1024) uint8_t smem[];
   using C = BCfg<D, KC, MODE, NBUF, RW>;
   constexpr uint32_t kTmemCols = C::kTmemCols;
@@ -152,7 +158,7 @@ bwd_tc_kernel(const __grid_constant__ BwdTcParams p) {
     for (int i = 0; i < C::kNumBars; ++i)
       mbar_init(bar(i), (i >= C::kBarPReady && i < C::kBarODone) ? kTile * C::kRowWgs
                         : (i == C::kBarRFull || (i >= C::kBarCFull && i < C::kBarCEmpty))
-                            ? kProducers : 1);
+                            ? (TMA ? 32 : kProducers) : 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 0) {
@@ -166,7 +172,82 @@ bwd_tc_kernel(const __grid_constant__ BwdTcParams p) {
   const uint32_t tmem = *tmem_slot;
   SA_LEAVE_IF_SKIPPED(reinterpret_cast<volatile int*>(smem + C::kOffMisc + 8), 0, tmem, kTmemCols)
 
-  if (warp >= 1 && warp < 4) {
+  if (warp >= 1 && warp < 4 && TMA) {
+    // ------------------------------------------------- tile loads by TMA (warp 1 alone)
+    // Rows and columns are consecutive tokens (no permutation, window by slots only), so a tile
+    // is D / 64 boxes of KC tokens x 64 columns per operand; tokens outside the sequence read
+    // zeros and are masked by the slot window.  Lane 0 posts the byte counts and the loads;
+    // for rows = keys the 32 lanes also fetch the per-query lse and delta of the columns.
+    // The token lists are not written: the one-sided rule does not look at them.
+    if (warp == 1) {
+      auto signal = [&](uint32_t mb) {
+        asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(mb) : "memory");
+      };
+      auto load_rows = [&](const CUtensorMap* tm, uint32_t dst, int tok, int head, int rows,
+                           uint32_t mb) {
+        for (int r = 0; r < rows; r += KC)
+#pragma unroll
+          for (int c = 0; c < D / 64; ++c)
+            tma_load_4d(dst + c * (rows * 128) + r * 128, tm, 64 * c, tok + r, head, b, mb);
+      };
+      if (lane == 0) {
+        mbar_expect_tx(bar(C::kBarRFull), 2 * C::kTileBytes);   // counts as this lane's arrival
+        load_rows(kKeys ? &tm_k : &tm_q, sbase + C::kOffR, r0, hr, kTile, bar(C::kBarRFull));
+        load_rows(kKeys ? &tm_v : &tm_dy, sbase + C::kOffR + C::kTileBytes, r0, hr, kTile,
+                  bar(C::kBarRFull));
+      } else {
+        mbar_arrive(bar(C::kBarRFull));
+      }
+      bool live = true;
+      int issued = 0;
+      for (int it = 0; it < iters && live; ++it) {
+        const int s = it % C::kStages;
+        const int j = kKeys ? it % T : it, gi = kKeys ? it / T : 0;
+        const int hq = kKeys ? hk * p.G + gi : hr;
+        if (it >= C::kStages)
+          live = mbar_wait(bar(C::kBarCEmpty + s), (it / C::kStages - 1) & 1u, gave_up, p.status);
+        live = __all_sync(0xffffffffu, live);
+        if (!live) break;
+        issued = it + 1;
+        const uint32_t colvec = sbase + C::kOffColVec + s * 2 * kTile * 4;
+        const uint32_t c1 = sbase + C::kOffC + s * 2 * C::kColBytes, c2 = c1 + C::kColBytes;
+        const uint32_t mb = bar(C::kBarCFull + s);
+        if (lane == 0) mbar_arrive(bar(C::kBarTokFull + s));
+        if (kKeys) {
+          const float* lse_h = p.lse + ((size_t)b * p.Hq + hq) * p.n;
+          const float* del_h = p.delta + ((size_t)b * p.Hq + hq) * p.n;
+          // (lanes 1-31: lane 0 arrives by posting the byte count, which does not wait for
+          // copies of its own)
+          for (int x = lane - 1; x < KC && lane > 0; x += 31) {
+            const int t0 = actual_slot(p, cstart + j * KC + x);
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(colvec + 4 * x), "l"(lse_h + t0) : "memory");
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(colvec + 4 * (kTile + x)), "l"(del_h + t0) : "memory");
+          }
+        }
+        if (lane == 0) {
+          mbar_expect_tx(mb, 2 * C::kColBytes);                 // this lane's arrival
+          load_rows(kKeys ? &tm_q : &tm_k, c1, cstart + j * KC, kKeys ? hq : hk, KC, mb);
+          load_rows(kKeys ? &tm_dy : &tm_v, c2, cstart + j * KC, kKeys ? hq : hk, KC, mb);
+        } else {
+          signal(mb);                                           // after this lane's small copies
+        }
+      }
+      asm volatile("cp.async.wait_all;" ::: "memory");
+      // loads that were started but never consumed (only after a failed wait) must land before
+      // the shared memory goes away: wait for them, again with a limit
+      if (lane == 0 && (!live || *gave_up)) {
+        for (int tries = 0; tries < 100000; ++tries) {
+          if (mbar_try(bar(C::kBarRFull), 0u)) break;
+          __nanosleep(100);
+        }
+        for (int u = issued > C::kStages ? issued - C::kStages : 0; u < issued; ++u)
+          for (int tries = 0; tries < 100000; ++tries) {
+            if (mbar_try(bar(C::kBarCFull + u % C::kStages), (u / C::kStages) & 1u)) break;
+            __nanosleep(100);
+          }
+      }
+    }
+  } else if (warp >= 1 && warp < 4) {
     // ---------------------------------------------------- gather producers (warps 1-3)
     constexpr int kCpr = D / 8;            // 16-byte pieces per row
     constexpr int kRpi = 32 / kCpr;        // rows per warp instruction
@@ -529,20 +610,31 @@ bwd_tc_kernel(const __grid_constant__ BwdTcParams p) {
 
 // ---------------------------------------------------------------------------- host
 
-template <int D, int KC, int NBUF, int RW>
-cudaError_t launch_branch(const BwdTcParams& p, cudaStream_t st) {
+template <int D, int KC, int NBUF, int RW, bool TMA>
+cudaError_t launch_branch_as(const BwdTcParams& p, const CUtensorMap* tm, cudaStream_t st) {
   using C0 = BCfg<D, KC, 0, NBUF, RW>;
   using C1 = BCfg<D, KC, 1, NBUF, RW>;
-  cudaError_t e = cudaFuncSetAttribute(bwd_tc_kernel<D, KC, 0, NBUF, RW>,
+  cudaError_t e = cudaFuncSetAttribute(bwd_tc_kernel<D, KC, 0, NBUF, RW, TMA>,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, C0::kBytes);
   if (e != cudaSuccess) return e;
-  e = cudaFuncSetAttribute(bwd_tc_kernel<D, KC, 1, NBUF, RW>,
+  e = cudaFuncSetAttribute(bwd_tc_kernel<D, KC, 1, NBUF, RW, TMA>,
                            cudaFuncAttributeMaxDynamicSharedMemorySize, C1::kBytes);
   if (e != cudaSuccess) return e;
-  bwd_tc_kernel<D, KC, 0, NBUF, RW><<<(unsigned)(p.B * p.Hq * p.n_tiles), C0::kThreads, C0::kBytes, st>>>(p);
-  bwd_tc_kernel<D, KC, 1, NBUF, RW><<<(unsigned)(p.B * p.Hkv * p.n_tiles), C1::kThreads, C1::kBytes, st>>>(p);
+  bwd_tc_kernel<D, KC, 0, NBUF, RW, TMA><<<(unsigned)(p.B * p.Hq * p.n_tiles), C0::kThreads, C0::kBytes, st>>>(
+      p, tm[0], tm[1], tm[2], tm[3]);
+  bwd_tc_kernel<D, KC, 1, NBUF, RW, TMA><<<(unsigned)(p.B * p.Hkv * p.n_tiles), C1::kThreads, C1::kBytes, st>>>(
+      p, tm[0], tm[1], tm[2], tm[3]);
   bump_launches(2);
   return cudaGetLastError();
+}
+
+// tm: tensor maps of q, k, v, dy with boxes of KC tokens when the branch's tiles come by TMA,
+// else null.
+template <int D, int KC, int NBUF, int RW>
+cudaError_t launch_branch(const BwdTcParams& p, const CUtensorMap* tm, cudaStream_t st) {
+  if (tm) return launch_branch_as<D, KC, NBUF, RW, true>(p, tm, st);
+  const CUtensorMap none[4] = {};
+  return launch_branch_as<D, KC, NBUF, RW, false>(p, none, st);
 }
 
 constexpr int kWideDefault = 1;   // shape for w > 128
@@ -591,13 +683,26 @@ cudaError_t launch_bwd_tc(const BwdArgs& a, cudaStream_t st) {
     p.scale2 = a.scale * kLog2e;
     for (int i = 0; i < 3; ++i) { p.qs[i] = a.qs[i]; p.ks[i] = a.ks[i]; }
     const int shape = bwd_shape(a.w);
+    // whole-tile TMA loads for the one-sided SWA branch (otherwise the gather serves it too)
+    CUtensorMap maps[4];
+    const CUtensorMap* tm = nullptr;
+    const int kc = shape == 2 ? 128 : 64;
+    if (x == 1 && mg.one_sided && debug_option(SA_DEBUG_SWA_TILE_LOADS) != 0 && aligned16(a.q) &&
+        aligned16(a.k) && aligned16(a.v) && aligned16(a.dy) &&
+        make_map_bhnd(&maps[0], a.q, a.B, a.Hq, a.n, a.d, a.qs, kc) &&
+        make_map_bhnd(&maps[1], a.k, a.B, a.Hkv, a.n, a.d, a.ks, kc) &&
+        make_map_bhnd(&maps[2], a.v, a.B, a.Hkv, a.n, a.d, a.ks, kc) &&
+        make_map_bhnd(&maps[3], a.dy, a.B, a.Hq, a.n, a.d, a.qs, kc))
+      tm = maps;
     cudaError_t e;
     if (a.d == 128)
-      e = shape == 0 ? launch_branch<128, 64, 1, 1>(p, st)
-          : shape == 1 ? launch_branch<128, 64, 2, 2>(p, st) : launch_branch<128, 128, 1, 2>(p, st);
+      e = shape == 0 ? launch_branch<128, 64, 1, 1>(p, tm, st)
+          : shape == 1 ? launch_branch<128, 64, 2, 2>(p, tm, st)
+                       : launch_branch<128, 128, 1, 2>(p, tm, st);
     else
-      e = shape == 0 ? launch_branch<64, 64, 1, 1>(p, st)
-          : shape == 1 ? launch_branch<64, 64, 2, 2>(p, st) : launch_branch<64, 128, 1, 2>(p, st);
+      e = shape == 0 ? launch_branch<64, 64, 1, 1>(p, tm, st)
+          : shape == 1 ? launch_branch<64, 64, 2, 2>(p, tm, st)
+                       : launch_branch<64, 128, 1, 2>(p, tm, st);
     if (e != cudaSuccess) return e;
   }
   return cudaSuccess;

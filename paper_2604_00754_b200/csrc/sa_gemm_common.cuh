@@ -76,11 +76,11 @@ inline bool make_map(CUtensorMap* tm, const void* base, int64_t rows, int64_t co
 }
 
 // bf16 tensor [B,H,n,d] with element strides s[0..2] (batch, head, token; d contiguous) as a
-// rank-4 map (d, token, head, batch), read in boxes of 64 columns x 128 tokens of one head
+// rank-4 map (d, token, head, batch), read in boxes of 64 columns x box_rows tokens of one head
 // with the 128-byte swizzle.  The token index is a dimension of its own, so a box that runs
 // past token n - 1 reads zeros there and never the rows that follow in memory.
 inline bool make_map_bhnd(CUtensorMap* tm, const void* base, int B, int H, int n, int d,
-                          const int64_t s[3]) {
+                          const int64_t s[3], int box_rows = 128) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   // the stride of a dimension of extent 1 is never used: any valid value will do
@@ -90,7 +90,7 @@ inline bool make_map_bhnd(CUtensorMap* tm, const void* base, int B, int H, int n
   const cuuint64_t dims[4] = {(cuuint64_t)d, (cuuint64_t)n, (cuuint64_t)H, (cuuint64_t)B};
   const cuuint64_t strides[3] = {(cuuint64_t)st[2] * 2, (cuuint64_t)st[1] * 2,
                                  (cuuint64_t)st[0] * 2};
-  const cuuint32_t box[4] = {64, 128, 1, 1};
+  const cuuint32_t box[4] = {64, (cuuint32_t)box_rows, 1, 1};
   const cuuint32_t estr[4] = {1, 1, 1, 1};
   return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,
             estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,

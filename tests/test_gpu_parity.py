@@ -160,6 +160,41 @@ def test_swa_branch_without_tma_tile_loads(debug_option):
     for fused in (False, True):
         for token_major in (False, True):
             test_gated_forward_both_combine_paths(bf, fused, token_major)
+    # the backward of the local branch loads its tiles the same two ways
+    for case in BWD_SMALL:
+        if case[6] & SWA_ONE_SIDED:
+            test_backward_small(*case, True, bf)
+
+
+def test_backward_swa_tiles_past_the_sequence_read_zeros():
+    """Gated backward on views of longer buffers whose tails hold NaN: the local branch's tile
+    loads must fill rows past token n - 1 with zeros (a NaN row would poison dK and dV of every
+    key of the tile through 0 * NaN)."""
+    B, Hq, Hkv, n, d, w, pad = 1, 4, 2, 389, 128, 200, 640
+    flags = CAUSAL | SWA_ONE_SIDED
+    q, k, v = draw((B, Hq, n, d), (B, Hkv, n, d), torch.bfloat16, seed=61)
+    g = torch.Generator().manual_seed(62)
+    dy = torch.randn(B, Hq, n, d, generator=g).to(torch.bfloat16)
+    lg = torch.randn(2, Hq, generator=g)
+    perm, inv, permc, invc = perms(61, 0, B, n)
+
+    def padded(t):
+        buf = torch.full((B, t.shape[1], pad, d), float("nan"), dtype=torch.bfloat16, device="cuda")
+        buf[:, :, :n] = t.cuda()
+        return buf[:, :, :n]
+    qd, kd, vd, dyd = padded(q), padded(k), padded(v), padded(dy)
+    mk = lambda like: torch.zeros((B, like.shape[1], pad, d), dtype=torch.bfloat16, device="cuda")[:, :, :n]
+    y, y_sa, y_swa, lse_sa, lse_swa = sa.sa_swa_gated_forward(
+        qd, kd, vd, perm, inv, lg.cuda(), w, flags, save_for_bwd=True,
+        out={"y": mk(q), "y_sa": mk(q), "y_swa": mk(q)})
+    dq, dk, dv, dg = sa.sa_backward(qd, kd, vd, perm, inv, lg.cuda(), y_sa, y_swa, lse_sa, lse_swa,
+                                    dyd, w, flags, out={"dq": mk(q), "dk": mk(k), "dv": mk(k)})
+    assert sa.sa_read_status() == 0
+    rdq, rdk, rdv, rdg = oracle.backward(as_f64(q), as_f64(k), as_f64(v), permc, invc,
+                                         lg.double().numpy(), as_f64(dy), w, flags)
+    for got, r, name in ((dq, rdq, "dq"), (dk, rdk, "dk"), (dv, rdv, "dv")):
+        assert torch.isfinite(got.float()).all(), name
+        close(got, r, torch.bfloat16, name)
 
 
 def test_cuda_core_kernels_on_tensor_core_shapes(debug_option):
