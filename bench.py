@@ -181,7 +181,7 @@ def main():
     ap.add_argument("--n", type=int, default=0,
                     help="override the sequence length (profiling captures on a smaller case)")
     ap.add_argument("--leg", default="step",
-                    choices=["step", "backward", "sa_fwd", "swa_fwd", "coverage"],
+                    choices=["step", "backward", "sa_fwd", "swa_fwd", "coverage", "gate"],
                     help="side measurements with their own JSON line (used for profiling): "
                          "backward = gated backward of the workload; sa_fwd / swa_fwd = that "
                          "branch's forward alone; coverage = the reach study of Prop. 2")
@@ -243,6 +243,9 @@ def main():
         return
     if args.leg in ("sa_fwd", "swa_fwd"):
         branch_leg(args, c, sa, torch, dev, perm, inv, ws, y, pk, rank)
+        return
+    if args.leg == "gate":
+        gate_leg(args, c, sa, torch, pk, rank)
         return
     if args.leg == "coverage":
         if rank == 0:
@@ -377,6 +380,30 @@ def branch_leg(args, c, sa, torch, dev, perm, inv, ws, y, pk, rank):
                           "tflops_nominal": tf, "frac_of_burst": tf / pk["bf16_tflops"],
                           "steps": args.steps, "warmup": args.warmup,
                           "config": workload_config(c), "dtype": "bf16", "data": "synthetic"}))
+
+
+def gate_leg(args, c, sa, torch, pk, rank):
+    """Projection gates of Eq. 5-6 at the workload's model width (Hq*d) over B*n rows: dual-path
+    forward and backward (what the counter summaries of those kernels are taken on)."""
+    dm, rows = c.Hq * c.d, c.B * c.n
+    gg = torch.Generator(device="cuda").manual_seed(17)
+    ya = torch.randn(rows, dm, generator=gg, device="cuda").bfloat16()
+    yb = torch.randn(rows, dm, generator=gg, device="cuda").bfloat16()
+    wa = (torch.randn(dm, dm, generator=gg, device="cuda") * dm ** -0.5).bfloat16()
+    wb = (torch.randn(dm, dm, generator=gg, device="cuda") * dm ** -0.5).bfloat16()
+    og = torch.empty_like(ya)
+    gbw = torch.empty(rows * dm * 8, dtype=torch.uint8, device="cuda")
+    f_ms = event_ms(lambda: sa.sa_gate_projection_forward(ya, wa, yb, wb, out=og), args.steps,
+                    args.warmup, torch)
+    b_ms = event_ms(lambda: sa.sa_gate_projection_backward(og, ya, wa, yb, wb, ws=gbw), args.steps,
+                    args.warmup, torch)
+    gfl = 2.0 * rows * dm * dm
+    if rank == 0:
+        print(json.dumps({"leg": "gate", "rows": rows, "dm": dm, "fwd_dual_ms": f_ms,
+                          "fwd_dual_tflops": 2 * gfl / (f_ms * 1e-3) / 1e12,
+                          "bwd_dual_ms": b_ms, "bwd_dual_tflops": 6 * gfl / (b_ms * 1e-3) / 1e12,
+                          "frac_of_burst_fwd": 2 * gfl / (f_ms * 1e-3) / 1e12 / pk["bf16_tflops"],
+                          "frac_of_burst_bwd": 6 * gfl / (b_ms * 1e-3) / 1e12 / pk["bf16_tflops"]}))
 
 
 def coverage_study(sa, torch, wl):
