@@ -303,11 +303,11 @@ def main():
     flops_branch = 4.0 * c.B * c.Hq * c.n * c.w * c.d
     achieved = flops_branch / (sa_kernel_ms * 1e-3) / 1e12
     # DRAM bytes of one SA-branch launch: dram__bytes_read.sum + dram__bytes_write.sum of one ncu
-    # capture of this kernel on this shape at n = 8192 (100.9 MB + 27.6 MB; the counter summary
+    # capture of this kernel on this shape at n = 8192 (100.9 MB + 26.5 MB; the counter summary
     # is under profiles/), scaled by n because every tensor grows in proportion to it.
     traffic = None
     if (c.B, c.Hq, c.Hkv, c.d, c.w) == (1, 32, 8, 128, 1024):
-        traffic = 128482304.0 * c.n / 8192
+        traffic = 127443200.0 * c.n / 8192
     sustained = args.steps * ms_per_step > 1500.0
     peak = pk["bf16_tflops_sustained"] if sustained else pk["bf16_tflops"]
     line = {
