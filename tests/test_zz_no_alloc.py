@@ -36,7 +36,7 @@ def test_static_scratch_matches_workspace_version_twice_in_a_row():
 def test_static_scratch_largest_and_too_large():
     perm, inv, want_perm, want_inv = both(11, 0, 1, 131072)
     assert torch.equal(perm, want_perm) and torch.equal(inv, want_inv)
-    B, n = 2, 131072                               # needs more than 5 MB of scratch: refused
+    B, n = 2, 131072                               # needs more than the 4 MiB built in: refused
     out = torch.empty(B, n, dtype=torch.int32, device="cuda")
     with pytest.raises(sa.SaError) as e:
         sa.sa_make_perm_static(1, 0, B, n, out, torch.empty_like(out))
