@@ -496,10 +496,14 @@ bwd_tc_kernel(const __grid_constant__ BwdTcParams p, const __grid_constant__ CUt
         uint32_t ds_pk[16], p_pk[16];
         auto chunk = [&](auto inter_c) {
         constexpr bool kInter = decltype(inter_c)::value;
+        // TMA tiles are the one-sided local branch: slots decide, the token lists are not even
+        // written, and their loads would only take shared-memory bandwidth from the products
+        constexpr bool kTok = !TMA;
 #pragma unroll
         for (int x = 0; x < 32; x += 4) {
           const int col = 32 * c + x;
-          const int4 ct = *reinterpret_cast<const int4*>(coltok + col);
+          int4 ct = make_int4(0, 0, 0, 0);
+          if (kTok) ct = *reinterpret_cast<const int4*>(coltok + col);
           float4 l4 = make_float4(lse2_r, lse2_r, lse2_r, lse2_r);
           float4 d4 = make_float4(delta_r, delta_r, delta_r, delta_r);
           if (kKeys) {
@@ -517,9 +521,9 @@ bwd_tc_kernel(const __grid_constant__ BwdTcParams p, const __grid_constant__ CUt
 #pragma unroll
           for (int y = 0; y < 4; y += 2) {
             const bool vis0 = (kInter || (uint32_t)(col + y - lo) <= span) &&
-                              (kKeys ? ctk[y] >= cmp : ctk[y] <= cmp);
+                              (!kTok || (kKeys ? ctk[y] >= cmp : ctk[y] <= cmp));
             const bool vis1 = (kInter || (uint32_t)(col + y + 1 - lo) <= span) &&
-                              (kKeys ? ctk[y + 1] >= cmp : ctk[y + 1] <= cmp);
+                              (!kTok || (kKeys ? ctk[y + 1] >= cmp : ctk[y + 1] <= cmp));
             const float2 a = __ffma2_rn(make_float2(__uint_as_float(sv[x + y]), __uint_as_float(sv[x + y + 1])),
                                         sc2, make_float2(-lv[y], -lv[y + 1]));
             const float2 ps = make_float2(vis0 ? exp2f(a.x) : 0.f, vis1 ? exp2f(a.y) : 0.f);   // P * scale
