@@ -117,7 +117,7 @@ struct BCfg {
 
 // MODE 0: rows are queries (dQ).  MODE 1: rows are keys (dK, dV).
 // TMA: the instantiation for the one-sided SWA branch, whose rows are consecutive tokens: one
-// warp loads whole tiles with cp.async.bulk.tensor (no multicast) instead of three warps
+// warp loads whole tiles with cp.async.bulk.tensor (every CTA its own) instead of three warps
 // gathering rows 16 bytes at a time, which is bound by the load/store unit.
 template <int D, int KC, int MODE, int NBUF, int RW, bool TMA>
 __global__ void __launch_bounds__(BCfg<D, KC, MODE, NBUF, RW>::kThreads,
