@@ -169,13 +169,17 @@ struct Cfg {
   static constexpr int kTok = D == 128 ? 3 : 8;
   static_assert((2 * kTok - kSlots) % 2 ? (2 * kTok - kSlots >= 1) : (2 * kTok - kSlots >= 4),
                 "token ring too short for the slot ring");
+  // Q buffers (two query tiles each).  With two (d = 64 leaves the room) the next item's Q is
+  // gathered, and its first scores are issued, while the row threads still finish this item:
+  // short items (narrow windows) otherwise idle a quarter of their time at every item start.
+  static constexpr int kQBufs = D == 128 ? 1 : 2;
   static constexpr int kOffQ = 0;
-  static constexpr int kOffRing = 2 * kTileBytes;
+  static constexpr int kOffRing = kQBufs * 2 * kTileBytes;
   static constexpr int kOffTok = kOffRing + kSlots * kTileBytes;
   static constexpr int kOffQTok = kOffTok + kTok * kTile * 4;   // tokens of the two query tiles
   static constexpr int kOffBar = kOffQTok + 2 * kTile * 4;
   // mbarriers, 8 bytes each
-  static constexpr int kBarQFull = 0, kBarQEmpty = 1, kBarSlotFull = 2,
+  static constexpr int kBarQFull = 0, kBarQEmpty = kQBufs, kBarSlotFull = 2 * kQBufs,
                        kBarSlotEmpty = kBarSlotFull + kSlots, kBarTokFull = kBarSlotEmpty + kSlots,
                        kBarSFull = kBarTokFull + kTok, kBarPReady = kBarSFull + 4,
                        kBarPvDone = kBarPReady + 4, kBarODone = kBarPvDone + 2,
@@ -225,7 +229,7 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
     for (int i = 0; i < C::kNumBars; ++i)
       mbar_init(bar(i), i >= C::kBarRowsTaken ? 64      // the two combining warps
                         : ((i >= C::kBarPReady && i < C::kBarPvDone) || i >= C::kBarRowsDone) ? kTile
-                        : (i == C::kBarQFull || (i >= C::kBarSlotFull && i < C::kBarSlotEmpty))
+                        : (i < C::kBarQEmpty || (i >= C::kBarSlotFull && i < C::kBarSlotEmpty))
                             ? (p.use_tma ? 1 : kProducers) : 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -286,14 +290,16 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
                     g.kstart + j * kTile, hk, b, mb);
           ++use;
           if (j == 0) {
-            if (it) live = mbar_wait(bar(C::kBarQEmpty), (it - 1) & 1u, gave_up, p.status);
+            const uint32_t qb = it % C::kQBufs;
+            if (it >= (uint32_t)C::kQBufs)
+              live = mbar_wait(bar(C::kBarQEmpty + qb), (it / C::kQBufs - 1) & 1u, gave_up, p.status);
             if (!live) break;
-            mbar_expect_tx(bar(C::kBarQFull), 2 * C::kTileBytes);
+            mbar_expect_tx(bar(C::kBarQFull + qb), 2 * C::kTileBytes);
             q_armed = it;
 #pragma unroll
             for (int t = 0; t < 2; ++t)
-              load_tile(&tm_q, sbase + C::kOffQ + t * C::kTileBytes, g.q0[t], g.hq[t], b,
-                        bar(C::kBarQFull));
+              load_tile(&tm_q, sbase + C::kOffQ + (2 * qb + t) * C::kTileBytes, g.q0[t], g.hq[t], b,
+                        bar(C::kBarQFull + qb));
           }
           if (use >= (uint32_t)C::kSlots)
             live = mbar_wait(bar(C::kBarSlotEmpty + use % C::kSlots), (use / C::kSlots - 1) & 1u,
@@ -317,7 +323,7 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
           }
         if (q_armed != 0xffffffffu)
           for (int tries = 0; tries < 100000; ++tries) {
-            if (mbar_try(bar(C::kBarQFull), q_armed & 1u)) break;
+            if (mbar_try(bar(C::kBarQFull + q_armed % C::kQBufs), (q_armed / C::kQBufs) & 1u)) break;
             __nanosleep(100);
           }
       }
@@ -565,7 +571,8 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
         }
         if (j == 0) {
           // ---- Q of this item, once the products of the previous item no longer read it
-          if (it) wait_free(bar(C::kBarQEmpty), (it - 1) & 1u);
+          if (it >= (uint32_t)C::kQBufs)
+            wait_free(bar(C::kBarQEmpty + it % C::kQBufs), (it / C::kQBufs - 1) & 1u);
           qtok[ptid] = tq0;
           qtok[ptid + 96] = tq1;
           if (ptid < 64) qtok[ptid + 192] = tq2;
@@ -573,8 +580,8 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
 #pragma unroll
           for (int t = 0; t < 2; ++t)
             gather(qg + b * p.qs[0] + g.hq[t] * p.qs[1], p.qs[2], qtok + t * kTile,
-                   sbase + C::kOffQ + t * C::kTileBytes);
-          if (ROPE) commit_group(); else signal(bar(C::kBarQFull));
+                   sbase + C::kOffQ + (2 * (it % C::kQBufs) + t) * C::kTileBytes);
+          if (ROPE) commit_group(); else signal(bar(C::kBarQFull + it % C::kQBufs));
         }
         // ---- V_j
         if (use >= (uint32_t)C::kSlots)
@@ -591,12 +598,12 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
           __syncwarp();
           rotate(ktok, k_dst);
           if (j == 0) {
-            rotate(qtok, sbase + C::kOffQ);
-            rotate(qtok + kTile, sbase + C::kOffQ + C::kTileBytes);
+            rotate(qtok, sbase + C::kOffQ + 2 * (it % C::kQBufs) * C::kTileBytes);
+            rotate(qtok + kTile, sbase + C::kOffQ + (2 * (it % C::kQBufs) + 1) * C::kTileBytes);
           }
           fence_proxy_async();
           mbar_arrive(k_bar);
-          if (j == 0) mbar_arrive(bar(C::kBarQFull));
+          if (j == 0) mbar_arrive(bar(C::kBarQFull + it % C::kQBufs));
         }
       }
     }
@@ -618,8 +625,8 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
       constexpr uint32_t kDescHi = (1024u >> 4) | (1u << 14) | (2u << 29);
       constexpr uint32_t kLoK = (16u >> 4) << 16;                          // K-major operands
       constexpr uint32_t kLoV = ((uint32_t)C::kChunkBytes >> 4) << 16;     // V: next 64 columns
-      const uint64_t q_desc0 = desc64(((sbase + C::kOffQ) >> 4) | kLoK, kDescHi);
-      const uint64_t q_desc1 = desc64(((sbase + C::kOffQ + C::kTileBytes) >> 4) | kLoK, kDescHi);
+      const uint64_t q_first = desc64(((sbase + C::kOffQ) >> 4) | kLoK, kDescHi);
+      uint64_t q_desc0 = q_first, q_desc1 = q_first + (C::kTileBytes >> 4);   // this item's Q tiles
       const uint32_t ring_lo = (sbase + C::kOffRing) >> 4;
       bool ok = true;
       uint32_t use = 0, it = 0;
@@ -661,7 +668,10 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
         active_halves(p, g.q0[1], g.valid[1], g.kstart, H, kShift, &first1, &last1);
         uint32_t started0 = 0, started1 = 0;
         // ring uses of this item: K_j = use + 2j, V_j = use + 2j + 1
-        ok = mbar_wait(bar(C::kBarQFull), it & 1u, gave_up, p.status);
+        const uint32_t qb = it % C::kQBufs;
+        q_desc0 = q_first + qb * (2 * C::kTileBytes >> 4);
+        q_desc1 = q_desc0 + (C::kTileBytes >> 4);
+        ok = mbar_wait(bar(C::kBarQFull + qb), (it / C::kQBufs) & 1u, gave_up, p.status);
         if (ok) ok = slot_wait(use);
         if (!ok) break;
         fence_proxy_async();
@@ -676,7 +686,7 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
           }
         }
         tc_commit(bar(C::kBarSlotEmpty + use % C::kSlots));
-        if (g.T == 1) tc_commit(bar(C::kBarQEmpty));
+        if (g.T == 1) tc_commit(bar(C::kBarQEmpty + qb));
         for (int j = 0; j < g.T && ok; ++j) {
           const uint32_t uv = use + 2 * j + 1, uk = use + 2 * j + 2;
           const bool more = j + 1 < g.T;
@@ -713,7 +723,7 @@ fwd_tc_kernel(const __grid_constant__ TcParams p, const __grid_constant__ CUtens
           // the slots free when the products issued so far have finished
           tc_commit(bar(C::kBarSlotEmpty + uv % C::kSlots));
           if (more) tc_commit(bar(C::kBarSlotEmpty + uk % C::kSlots));
-          if (j + 2 == g.T) tc_commit(bar(C::kBarQEmpty));
+          if (j + 2 == g.T) tc_commit(bar(C::kBarQEmpty + qb));
         }
         use += 2 * g.T;
       }
