@@ -55,6 +55,7 @@ ROPE_CASES = [
     (1, 8, 2, 1153, 64, 128, CAUSAL),                  # group of 4: two heads share a stream
     (1, 3, 3, 700, 128, 96, 0),                        # odd group: two slot tiles per item
     (1, 2, 2, 515, 128, 300, CAUSAL | LINEAR_WINDOW),
+    (2, 8, 2, 6000, 64, 96, CAUSAL),                   # several items per CTA: both Q buffers turn over
 ]
 
 
