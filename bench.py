@@ -490,8 +490,8 @@ def extras(args, c, wl, sa, torch, dev, host, perm, inv, ws, y, pk):
                   "h2d_bytes_per_step": sum(host[x].numel() for x in ("q", "k", "v")) * elt
                                         + hg.numel() * 4,
                   "d2h_bytes_per_step": hy.numel() * elt,
-                  "api": "sa_swa_gated_forward_host (C ABI, host pointers), 8 KV-head groups x 2 "
-                         "query-head parts on 3 streams"}
+                  "api": "sa_swa_gated_forward_host (C ABI, host pointers), 8 KV-head groups, the "
+                         "first and last cut in 2 query-head parts, on 3 streams"}
     del hws
     torch.cuda.empty_cache()
 

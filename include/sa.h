@@ -168,8 +168,9 @@ sa_status sa_swa_gated_forward(const sa_problem* p, const void* q, const void* k
  * HOST memory: q, k, v, y are host pointers to contiguous [B,H,n,d] tensors of p->dtype
  * (p's stride fields are ignored), gate_logits a host pointer to fp32 [2,Hq]; pinned memory
  * lets the copies overlap the kernels, pageable memory works but serialises.  The KV heads
- * travel through the GPU in n_groups contiguous ranges (a range of one KV head in q_parts
- * ranges of its query heads when they divide evenly), on three internal streams: copy in,
+ * travel through the GPU in n_groups contiguous ranges (the first and the last range, when
+ * they hold one KV head, in q_parts ranges of its query heads if those divide evenly: the
+ * ends of the pipeline are what cannot overlap), on three internal streams: copy in,
  * compute, copy out.  The permutation is drawn from (seed, layer) as in sa_make_perm and
  * shared by all ranges; every range is one sa_swa_gated_forward call given scratch, so the
  * result has the bits of that call.

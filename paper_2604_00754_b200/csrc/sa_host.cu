@@ -19,9 +19,11 @@ constexpr int kMaxPieces = 256;
 
 struct Piece { int ka, kb, qa, qb, with_kv; };
 
-// KV heads in at most n_groups contiguous ranges; a range of one KV head is cut further into
-// q_parts ranges of query heads when they divide evenly (only the first carries K/V): smaller
-// first and last pieces shorten the parts of the pipeline that cannot overlap.
+// KV heads in at most n_groups contiguous ranges.  The first and the last range, when they hold
+// one KV head, are cut further into q_parts ranges of query heads if those divide evenly (only
+// the first part carries K/V): the copy in of the first piece and the kernels and copy out of
+// the last one are what cannot overlap, so those pieces are small; the pieces in between are
+// large, because every piece costs launches and events.
 int plan(int Hq, int Hkv, int n_groups, int q_parts, Piece* out, int max_out) {
   if (Hq < 1 || Hkv < 1 || Hq % Hkv != 0 || !out) return -1;
   const int G = Hq / Hkv;
@@ -30,7 +32,8 @@ int plan(int Hq, int Hkv, int n_groups, int q_parts, Piece* out, int max_out) {
   for (int i = 0; i < n_groups; ++i) {
     const int a = (int)((int64_t)i * Hkv / n_groups), b = (int)((int64_t)(i + 1) * Hkv / n_groups);
     if (b <= a) continue;
-    if (b - a == 1 && q_parts > 1 && G % q_parts == 0) {
+    const bool edge = i == 0 || i == n_groups - 1;
+    if (edge && b - a == 1 && q_parts > 1 && G % q_parts == 0) {
       const int step = G / q_parts;
       for (int j = 0; j < q_parts; ++j) {
         if (cnt >= max_out) return -1;

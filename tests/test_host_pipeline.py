@@ -21,11 +21,15 @@ def test_head_groups_cover_every_head_once():
 
 
 def test_split_query_heads_keeps_coverage_and_kv_ownership():
+    # the first and the last KV head are cut by query heads, the ones in between stay whole
     g = sab.host_forward_plan(32, 8, 8, 2)
-    assert len(g) == 16
-    assert [x[2:4] for x in g] == [(2 * i, 2 * i + 2) for i in range(16)]
-    assert [x[4] for x in g] == [True, False] * 8          # K/V travel with the first part only
+    assert [x[2:4] for x in g] == [(0, 2), (2, 4)] + [(4 * i, 4 * i + 4) for i in range(1, 7)] + \
+        [(28, 30), (30, 32)]
+    assert [x[4] for x in g] == [True, False] + [True] * 6 + [True, False]   # K/V with the first part
     assert all(kb - ka == 1 for ka, kb, *_ in g)
+    g = sab.host_forward_plan(32, 8, 8, 4)
+    assert len(g) == 14 and [x[2:4] for x in g][-4:] == [(28, 29), (29, 30), (30, 31), (31, 32)]
+    assert sab.host_forward_plan(4, 1, 1, 2) == [(0, 1, 0, 2, True), (0, 1, 2, 4, False)]
     # ranges with several KV heads, or an odd number of query heads per KV head, stay whole
     assert sab.host_forward_plan(8, 4, 2, 2) == [(0, 2, 0, 4, True), (2, 4, 4, 8, True)]
     assert sab.host_forward_plan(3, 1, 1, 2) == [(0, 1, 0, 3, True)]
