@@ -93,7 +93,8 @@ bool carve(const sa_problem* p, Carve* c) {
   c->v = o; o += align256(kb);
   c->y = o; o += align256(qb);
   c->scratch = o; o += align256(qb);
-  c->gate = o; o += align256((size_t)2 * p->Hq * sizeof(float));
+  // the logits as they come ([2, Hq]), then one contiguous [2, heads] block per piece
+  c->gate = o; o += 2 * align256((size_t)2 * p->Hq * sizeof(float));
   c->perm = o; o += align256((size_t)p->B * p->n * sizeof(int32_t));
   c->inv = o; o += align256((size_t)p->B * p->n * sizeof(int32_t));
   c->perm_ws = o; o += align256(make_perm_ws_bytes(p->B, p->n));
@@ -152,7 +153,8 @@ sa_status sa_swa_gated_forward_host(const sa_problem* p, const void* q, const vo
   const size_t es = p->dtype == SA_BF16 ? 2 : 4;
   const size_t head_bytes = (size_t)p->n * p->d * es;
   char *dq = base + c.q, *dk = base + c.k, *dv = base + c.v, *dyv = base + c.y;
-  float* dgate = (float*)(base + c.gate);
+  float* dgate_all = (float*)(base + c.gate);
+  float* dgate = (float*)(base + c.gate + align256((size_t)2 * p->Hq * sizeof(float)));
   int32_t* dperm = (int32_t*)(base + c.perm);
   int32_t* dinv = (int32_t*)(base + c.inv);
   cudaStream_t cur = (cudaStream_t)stream;
@@ -165,16 +167,17 @@ sa_status sa_swa_gated_forward_host(const sa_problem* p, const void* q, const vo
   chk(cudaStreamWaitEvent(pipe->s_run, pipe->ev_start, 0));
   chk(cudaStreamWaitEvent(pipe->s_out, pipe->ev_start, 0));
 
-  // copy in: the logits of each piece as one contiguous [2, heads] block, then its heads
+  // copy in: all logits in one small copy (a copy of a few bytes holds the copy engine as long
+  // as one of a few hundred kilobytes, and two per piece stood between the large ones), then
+  // the heads of each piece; the [2, heads] block of a piece is cut out on the compute stream
+  chk(cudaMemcpyAsync(dgate_all, gate_logits, (size_t)2 * p->Hq * sizeof(float),
+                      cudaMemcpyHostToDevice, pipe->s_in));
   size_t gate_off = 0;
   size_t gate_at[kMaxPieces];
   for (int i = 0; i < cnt && ok; ++i) {
     const Piece& g = pieces[i];
     const int hq = g.qb - g.qa;
     gate_at[i] = gate_off;
-    for (int x = 0; x < 2; ++x)
-      chk(cudaMemcpyAsync(dgate + gate_off + (size_t)x * hq, gate_logits + (size_t)x * p->Hq + g.qa,
-                          hq * sizeof(float), cudaMemcpyHostToDevice, pipe->s_in));
     gate_off += (size_t)2 * hq;
     for (int b = 0; b < p->B; ++b) {   // one contiguous block per sequence and tensor
       if (g.with_kv) {
@@ -196,6 +199,9 @@ sa_status sa_swa_gated_forward_host(const sa_problem* p, const void* q, const vo
   for (int i = 0; i < cnt && ok && st == SA_OK; ++i) {
     const Piece& g = pieces[i];
     chk(cudaStreamWaitEvent(pipe->s_run, pipe->ev_in[i], 0));
+    chk(cudaMemcpy2DAsync(dgate + gate_at[i], (size_t)(g.qb - g.qa) * sizeof(float), dgate_all + g.qa,
+                          (size_t)p->Hq * sizeof(float), (size_t)(g.qb - g.qa) * sizeof(float), 2,
+                          cudaMemcpyDeviceToDevice, pipe->s_run));
     sa_problem gp = dp;                     // a view of the whole-size buffers: same strides
     gp.Hq = g.qb - g.qa;
     gp.Hkv = g.kb - g.ka;
