@@ -484,7 +484,7 @@ def extras(args, c, wl, sa, torch, dev, host, perm, inv, ws, y, pk):
         sa.sa_swa_gated_forward_host(host["q"], host["k"], host["v"], hg, hy, c.w, c.flags,
                                      c.seed, layer[0], hws, n_groups=8, q_parts=2)
         layer[0] += 1
-    e2e_ms = event_ms(e2e_step, it, 2, torch)
+    e2e_ms = event_ms(e2e_step, it, 3, torch)
     elt = host["q"].element_size()
     res["e2e"] = {"value": c.B * c.n / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms,
                   "h2d_bytes_per_step": sum(host[x].numel() for x in ("q", "k", "v")) * elt
@@ -508,7 +508,7 @@ def extras(args, c, wl, sa, torch, dev, host, perm, inv, ws, y, pk):
             r = sa.sa_backward(q, k, v, perm, inv, lg, sv[1], sv[2], sv[3], sv[4], dyb, c.w,
                                c.flags, ws=bws3, out=bo)
             bo.update(zip(("dq", "dk", "dv", "dgate"), r))
-        bms = event_ms(bwd_main, max(3, it // 2), 2, torch)
+        bms = event_ms(bwd_main, max(3, it // 2), 3, torch)
         bfl = 2 * 2.5 * flops
         res["backward_%s" % c.name.split("_")[0]] = {
             "gated_bwd_ms": bms, "tokens_per_s": c.B * c.n / (bms * 1e-3),
@@ -581,7 +581,7 @@ def extras(args, c, wl, sa, torch, dev, host, perm, inv, ws, y, pk):
             sa.sa_make_perm(c4.seed, l, c4.B, c4.n, perm=p4, inv=i4, ws=ws4)
             sa.sa_swa_gated_forward(t4["q"], t4["k"], t4["v"], p4, i4, t4["gate_logits"], c4.w,
                                     c4.flags, out={"y": y4}, ws=g4)
-    ms4 = event_ms(prefill, 2, 1, torch)
+    ms4 = event_ms(prefill, 2, 3, torch)
     fl4 = 2 * 4.0 * c4.B * c4.Hq * c4.n * c4.w * c4.d * c4.layers
     res["C4_prefill_48_layers"] = {
         "total_ms": ms4, "ms_per_layer": ms4 / c4.layers,
@@ -612,8 +612,8 @@ def extras(args, c, wl, sa, torch, dev, host, perm, inv, ws, y, pk):
                            saved["y_swa"], saved["lse_sa"], saved["lse_swa"], t5["dy"], c5.w,
                            c5.flags, ws=bws, out=bout)
         bout.update(zip(("dq", "dk", "dv", "dgate"), r))
-    f5 = event_ms(fwd5, it, 2, torch)
-    b5 = event_ms(bwd5, it, 2, torch)
+    f5 = event_ms(fwd5, it, 3, torch)
+    b5 = event_ms(bwd5, it, 3, torch)
     fl5 = 2 * 4.0 * c5.B * c5.Hq * c5.n * c5.w * c5.d
     ws5 = torch.empty(sa.sa_workspace_bytes(sa.SaProblem(B=c5.B, n=c5.n), sa.OP_MAKE_PERM),
                       dtype=torch.uint8, device="cuda")
@@ -623,7 +623,7 @@ def extras(args, c, wl, sa, torch, dev, host, perm, inv, ws, y, pk):
             sa.sa_make_perm(c5.seed, l, c5.B, c5.n, perm=p5, inv=i5, ws=ws5)
             fwd5()
             bwd5()
-    s5 = event_ms(step5, 3, 1, torch)
+    s5 = event_ms(step5, 3, 3, torch)
     bytes5 = 15 * 2.0 * c5.B * c5.Hq * c5.n * c5.d          # 15 tensor passes of 50.3 MB per layer
     res["pretrain_layer_C5"] = {
         "gated_fwd_ms": f5, "bwd_ms": b5, "tokens_per_s_fwd_bwd": c5.B * c5.n / ((f5 + b5) * 1e-3),
@@ -656,7 +656,7 @@ def extras(args, c, wl, sa, torch, dev, host, perm, inv, ws, y, pk):
             r = sa.sa_backward(d3["q"], d3["k"], d3["v"], p3, i3, None, y3, None, l3, None,
                                d3["dy"], c3.w, c3.flags, ws=w3, out=o3)
             o3.update(zip(("dq", "dk", "dv", "dgate"), r))
-        t3[str(n3)] = {"sa_fwd_bwd_ms": event_ms(fb3, 3, 2, torch),
+        t3[str(n3)] = {"sa_fwd_bwd_ms": event_ms(fb3, 3, 3, torch),
                        "paper_a100_flexattention_ms": paper_ms[n3]}
         # the table's other column: full causal attention, here the same kernels with the
         # identity permutation and a window that covers the whole sequence
@@ -668,7 +668,7 @@ def extras(args, c, wl, sa, torch, dev, host, perm, inv, ws, y, pk):
             r = sa.sa_backward(d3["q"], d3["k"], d3["v"], ident, ident, None, y3, None, l3, None,
                                d3["dy"], wfull, sa.CAUSAL, ws=w3, out=o3)
             o3.update(zip(("dq", "dk", "dv", "dgate"), r))
-        t3[str(n3)]["full_attention_fwd_bwd_ms"] = event_ms(full3, 2, 1, torch)
+        t3[str(n3)]["full_attention_fwd_bwd_ms"] = event_ms(full3, 2, 3, torch)
         t3[str(n3)]["paper_a100_full_attention_ms"] = paper_full_ms[n3]
         del d3, y3, l3, w3, o3
         torch.cuda.empty_cache()
@@ -695,7 +695,7 @@ def extras(args, c, wl, sa, torch, dev, host, perm, inv, ws, y, pk):
         "single_frac_of_burst": gfl / (g1 * 1e-3) / 1e12 / pk["bf16_tflops"]}
     # and their backward (dz, dy, dw: three products per path)
     gbw = torch.empty(rows_g * dm * 8, dtype=torch.uint8, device="cuda")
-    gb2 = event_ms(lambda: sa.sa_gate_projection_backward(og, ya, wa, yb, wb, ws=gbw), 3, 2, torch)
+    gb2 = event_ms(lambda: sa.sa_gate_projection_backward(og, ya, wa, yb, wb, ws=gbw), 3, 3, torch)
     res["gate_projection"].update({
         "bwd_dual_ms": gb2, "bwd_dual_tflops": 6 * gfl / (gb2 * 1e-3) / 1e12,
         "bwd_dual_frac_of_burst": 6 * gfl / (gb2 * 1e-3) / 1e12 / pk["bf16_tflops"]})
